@@ -1,0 +1,76 @@
+"""Cross-attention with log2-quantized softmax scores, Sec. 3.3 (Eq. 3, Eq. 8, Eq. 9).
+
+Test infrastructure only; see the package docstring.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+from .quantizers import log_quantize, log_dequantize
+
+PER_PROMPT, PER_PROMPT_HEAD, PER_CALL = 0, 1, 2
+FLT_MIN = float(np.finfo(np.float32).tiny)
+
+
+def softmax_scores(Q, K):
+    """Eq. 3: A = softmax_j(Q_i . K_j / sqrt(d)), fp64.  Q [B, nq, H, d], K [B, nk, H, d] -> A [B, H, nq, nk]."""
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    d = Q.shape[-1]
+    logits = np.einsum("bqhd,bkhd->bhqk", Q, K) / np.sqrt(np.float64(d))
+    logits -= logits.max(axis=-1, keepdims=True)
+    e = np.exp(logits)
+    return e / e.sum(axis=-1, keepdims=True)
+
+
+def prompt_scale(A, gran=PER_PROMPT):
+    """The dynamic scale of Eq. 8: s = max(A[:, 1:]), the largest score off the <start> column.
+
+    Eq. 8 writes A as one n_q x n_k map while the text ties the scale to the
+    input prompt; reading (parity unpinned): PER_PROMPT takes the maximum over
+    all heads, queries and keys j >= 1 of one prompt.  PER_PROMPT_HEAD and
+    PER_CALL are the narrower and wider scopes.  Returns s broadcastable to A
+    [B, H, nq, nk]; a zero maximum is raised to the smallest normal fp32.
+    """
+    rest = A[..., 1:]
+    if gran == PER_PROMPT:
+        s = rest.max(axis=(1, 2, 3), keepdims=True)
+    elif gran == PER_PROMPT_HEAD:
+        s = rest.max(axis=(2, 3), keepdims=True)
+    else:
+        s = rest.max(keepdims=True)
+    return np.maximum(s, FLT_MIN)
+
+
+def cross_attn_logq(Q, K, V, bits, gran=PER_PROMPT, fixed_scale=None):
+    """Attention-aware quantization (Eq. 8, Eq. 9), fp64 throughout.
+
+    Steps in the paper's order: full-precision softmax (Eq. 3); scale s from the
+    scores off the <start> column (or `fixed_scale`, the static variant of the
+    ablation in Table 3(c)); log2 codes of columns j >= 1 (Eq. 8, which is Eq. 2
+    with that s); A_hat = [A[:, 0], s 2^-codes] with column 0 untouched; the
+    product A_hat V as the sum of the <start> term and the quantized rest
+    (Eq. 9).  No re-normalisation of A_hat (none is described) and V stays as
+    given (V_hat = V on this path).  Returns O [B, nq, H, d], codes
+    [B, H, nq, nk-1], s (broadcast shape), A.
+    """
+    A = softmax_scores(Q, K)
+    V = np.asarray(V, dtype=np.float64)
+    if A.shape[-1] < 2:
+        raise ValueError("n_k < 2: no score off the <start> column to scale by")
+    if fixed_scale is None:
+        s = prompt_scale(A, gran)
+    else:
+        s = np.maximum(np.asarray(fixed_scale, dtype=np.float64).reshape(-1, 1, 1, 1), FLT_MIN)
+    s_full = np.broadcast_to(s, A.shape[:-1] + (1,))
+    codes = log_quantize(A[..., 1:], s_full, bits)
+    A_hat_rest = log_dequantize(codes, s_full)
+    O = (np.einsum("bhq,bhd->bqhd", A[..., 0], V[:, 0])
+         + np.einsum("bhqk,bkhd->bqhd", A_hat_rest, V[:, 1:]))
+    return O, codes, s, A
+
+
+def attention_reference(Q, K, V):
+    """Plain softmax attention softmax(Q K^T / sqrt(d)) V in fp64 (no quantization)."""
+    A = softmax_scores(Q, K)
+    return np.einsum("bhqk,bkhd->bqhd", A, np.asarray(V, dtype=np.float64))

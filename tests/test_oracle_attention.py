@@ -1,0 +1,126 @@
+"""Pins for the oracle's log-quantized cross-attention (Eq. 3, Eq. 8, Eq. 9)."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import attention as oa
+from paper_2501_04304_b200 import synth
+
+
+def _inputs(seed=0, B=2, H=2, nq=24, nk=9, d=8):
+    return synth.attention_inputs(seed, B, H, nq, nk, d, ctx_dim=32)
+
+
+def test_softmax_matches_library_sdpa():
+    torch = pytest.importorskip("torch")
+    Q, K, V = _inputs()
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(Q.astype(np.float64)).permute(0, 2, 1, 3),
+        torch.from_numpy(K.astype(np.float64)).permute(0, 2, 1, 3),
+        torch.from_numpy(V.astype(np.float64)).permute(0, 2, 1, 3)).permute(0, 2, 1, 3).numpy()
+    got = oa.attention_reference(Q, K, V)
+    assert np.max(np.abs(got - ref)) < 1e-12
+    A = oa.softmax_scores(Q, K)
+    assert np.allclose(A.sum(-1), 1.0, atol=1e-14)
+
+
+def test_brute_force_tiny():
+    Q, K, V = _inputs(seed=1, B=1, H=1, nq=16, nk=3, d=8)
+    O, codes, s, A = oa.cross_attn_logq(Q, K, V, 8)
+    Qf, Kf, Vf = Q.astype(float), K.astype(float), V.astype(float)
+    P = [[0.0] * 3 for _ in range(16)]
+    for i in range(16):
+        l = [sum(Qf[0, i, 0, c] * Kf[0, j, 0, c] for c in range(8)) / math.sqrt(8) for j in range(3)]
+        m = max(l)
+        e = [math.exp(v - m) for v in l]
+        P[i] = [v / sum(e) for v in e]
+    smax = max(P[i][j] for i in range(16) for j in (1, 2))
+    assert abs(float(s.ravel()[0]) - smax) < 1e-15
+    for i in range(16):
+        out = [P[i][0] * Vf[0, 0, 0, c] for c in range(8)]
+        for j in (1, 2):
+            q = min(max(round(-math.log2(P[i][j] / smax)), 0), 255)
+            assert q == codes[0, 0, i, j - 1]
+            for c in range(8):
+                out[c] += smax * 2.0 ** -q * Vf[0, j, 0, c]
+        assert np.allclose(O[0, i, 0], out, rtol=1e-12, atol=1e-15)
+
+
+@pytest.mark.parametrize("bits", [4, 6, 8])
+def test_structure_of_quantized_scores(bits):
+    Q, K, V = _inputs(seed=2)
+    B, nq, H, d = Q.shape
+    nk = K.shape[1]
+    O, codes, s, A = oa.cross_attn_logq(Q, K, V, bits)
+    assert codes.min() >= 0 and codes.max() <= 2 ** bits - 1
+    # the <start> column passes through unchanged: V = indicator of key 0 gives back A[:, 0] bit for bit
+    V0 = np.zeros_like(V, dtype=np.float64); V0[:, 0] = 1.0
+    O0, *_ = oa.cross_attn_logq(Q, K, V0, bits)
+    assert np.array_equal(O0[..., 0], A[..., 0].transpose(0, 2, 1))
+    # per prompt: the largest off-<start> score has code 0 and de-quantizes to exactly s
+    for b in range(B):
+        rest = A[b, :, :, 1:]
+        h, i, j = np.unravel_index(np.argmax(rest), rest.shape)
+        assert float(s[b].ravel()[0]) == rest[h, i, j]
+        assert codes[b, h, i, j] == 0
+        Vj = np.zeros_like(V, dtype=np.float64); Vj[:, j + 1] = 1.0
+        Oj, *_ = oa.cross_attn_logq(Q, K, Vj, bits)
+        assert Oj[b, i, h, 0] == rest[h, i, j]
+    # un-clamped entries are within a factor sqrt(2) of the score
+    s_full = np.broadcast_to(s, codes.shape[:-1] + (1,))
+    A_hat = np.ldexp(s_full, -codes)
+    ok = codes < 2 ** bits - 1
+    ratio = (A_hat / A[..., 1:])[ok]
+    assert ratio.min() >= 2 ** -0.5 * (1 - 1e-12) and ratio.max() <= 2 ** 0.5 * (1 + 1e-12)
+
+
+def test_codes_invariant_to_row_logit_shift():
+    Q, K, V = _inputs(seed=3)
+    _, c0, _, _ = oa.cross_attn_logq(Q, K, V, 8)
+    delta = np.random.default_rng(0).standard_normal(K.shape[-1]) * 0.25
+    K2 = K.astype(np.float64) + delta            # adds q_i . delta to every logit of row i
+    _, c1, _, _ = oa.cross_attn_logq(Q, K2, V, 8)
+    assert (c0 != c1).mean() < 1e-3 and np.abs(c0 - c1).max() <= 1
+
+
+def test_lossless_case_equals_textbook_attention():
+    """Logits that are integer multiples of ln 2 make every off-<start> score an exact power of
+    two times the scale: codes are exact and the output is plain softmax attention."""
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(4)
+    B, H, nq, nk, d = 2, 2, 12, 7, 4
+    Q = np.zeros((B, nq, H, d)); Q[..., 0] = math.sqrt(d) * math.log(2.0)
+    K = np.zeros((B, nk, H, d)); K[..., 0] = rng.integers(-6, 1, (B, nk, 1))      # same keys in every head: equal row sums
+    K[:, 1, :, 0] = 0                      # the off-<start> maximum
+    K[:, 0, :, 0] = 3                      # a dominant <start> column
+    V = rng.standard_normal((B, nk, H, d))
+    O, codes, s, A = oa.cross_attn_logq(Q, K, V, 8)
+    assert np.array_equal(codes, np.broadcast_to(-K[:, 1:, :, 0].transpose(0, 2, 1)[:, :, None, :], codes.shape))
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(Q).permute(0, 2, 1, 3), torch.from_numpy(K).permute(0, 2, 1, 3),
+        torch.from_numpy(V).permute(0, 2, 1, 3)).permute(0, 2, 1, 3).numpy()
+    assert np.max(np.abs(O - ref)) < 1e-13
+
+
+def test_scale_granularity_and_fixed_scale():
+    Q, K, V = _inputs(seed=5)
+    A = oa.softmax_scores(Q, K)
+    sp = oa.prompt_scale(A, oa.PER_PROMPT)
+    sh = oa.prompt_scale(A, oa.PER_PROMPT_HEAD)
+    sc = oa.prompt_scale(A, oa.PER_CALL)
+    assert np.array_equal(sp.ravel(), sh.max(axis=1).ravel())
+    assert sc.ravel()[0] == sp.max()
+    # static variant with the dynamic scale passed in reproduces the dynamic result
+    O, codes, s, _ = oa.cross_attn_logq(Q, K, V, 8)
+    O2, codes2, _, _ = oa.cross_attn_logq(Q, K, V, 8, fixed_scale=sp.ravel())
+    assert np.array_equal(codes, codes2) and np.array_equal(O, O2)
+    with pytest.raises(ValueError):
+        oa.cross_attn_logq(Q, K[:, :1], V[:, :1], 8)
+
+
+def test_four_bit_agrees_with_eight_bit_below_saturation():
+    Q, K, V = _inputs(seed=6)
+    _, c8, _, _ = oa.cross_attn_logq(Q, K, V, 8)
+    _, c4, _, _ = oa.cross_attn_logq(Q, K, V, 4)
+    assert np.array_equal(c4[c8 <= 15], c8[c8 <= 15]) and np.all(c4[c8 > 15] == 15)
