@@ -54,7 +54,8 @@ def group_params(lo, hi, b):
         x = min x maps to code 0;
       * a constant group (hi == lo) gets the floor scale 1e-8;
       * arithmetic is IEEE fp32, in this order: s = (hi - lo) * 2^-b,
-        inv_s = 1 / s, Z = rint(-lo * inv_s).
+        inv_s = 1 / s, Z = rint(clamp(-lo * inv_s, -2^30, 2^30)); the clamp only
+        matters for a constant group far from zero, where it keeps Z an int32.
     Returns (s, inv_s, Z) as (float32, float32, int).
     """
     lo = F32(lo)
@@ -63,7 +64,7 @@ def group_params(lo, hi, b):
     if not s > MIN_SCALE:
         s = MIN_SCALE
     inv_s = F32(F32(1.0) / s)
-    Z = int(np.rint(F32(-lo * inv_s)))
+    Z = int(np.rint(np.clip(F32(-lo * inv_s), F32(-2.0 ** 30), F32(2.0 ** 30))))
     return s, inv_s, Z
 
 
@@ -74,7 +75,7 @@ def group_params_array(lo, hi, b):
     s = ((hi - lo).astype(F32) * F32(2.0 ** -b)).astype(F32)
     s = np.where(s > MIN_SCALE, s, MIN_SCALE).astype(F32)
     inv_s = (F32(1.0) / s).astype(F32)
-    Z = np.rint((-lo * inv_s).astype(F32)).astype(np.int32)
+    Z = np.rint(np.clip((-lo * inv_s).astype(F32), F32(-2.0 ** 30), F32(2.0 ** 30))).astype(np.int32)
     return s, inv_s, Z
 
 

@@ -1,0 +1,211 @@
+// Shared host/device helpers of the DGQ library: status word, checked CUDA calls,
+// mbarrier / TMA / tcgen05 PTX wrappers with bounded waits.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <cuda.h>
+
+#include <atomic>
+#include <cstdint>
+#include <cstring>
+#include <vector>
+
+#include "../../include/dgq.h"
+
+namespace dgq {
+
+// First error recorded by any kernel on this device since the last dgq_device_status().
+__device__ int g_status_word = 0;
+
+static std::atomic<uint64_t> g_launches{0};
+
+__device__ __forceinline__ void record_error(int code) { atomicCAS(&g_status_word, 0, code); }
+
+#define DGQ_CUDA_OK(expr)                        \
+  do {                                           \
+    cudaError_t e__ = (expr);                    \
+    if (e__ != cudaSuccess) return DGQ_ERR_CUDA; \
+  } while (0)
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ------------------------------------------------------------------ ordered-int encoding of floats
+// Monotone map float -> int so that integer atomicMin / atomicMax order like the floats.
+__host__ __device__ __forceinline__ int float_to_ordered(float f) {
+#ifdef __CUDA_ARCH__
+  int b = __float_as_int(f);
+#else
+  int b;
+  std::memcpy(&b, &f, 4);
+#endif
+  return b >= 0 ? b : (b ^ 0x7FFFFFFF);
+}
+__host__ __device__ __forceinline__ float ordered_to_float(int k) {
+  int b = k >= 0 ? k : (k ^ 0x7FFFFFFF);
+#ifdef __CUDA_ARCH__
+  return __int_as_float(b);
+#else
+  float f;
+  std::memcpy(&f, &b, 4);
+  return f;
+#endif
+}
+
+// ------------------------------------------------------------------ Eq. 6 in the fixed fp32 order
+// s = (hi - lo) * 2^-b floored at 1e-8, inv_s = 1 / s (IEEE division),
+// Z = rint(clamp(-lo * inv_s, -2^30, 2^30)).
+__host__ __device__ __forceinline__ void group_params(float lo, float hi, int bits, float& s, float& inv_s,
+                                                       int& Z) {
+#ifdef __CUDA_ARCH__
+  float w = __fmul_rn(__fsub_rn(hi, lo), __int_as_float((127 - bits) << 23));
+  s = w > 1e-8f ? w : 1e-8f;
+  inv_s = __fdiv_rn(1.0f, s);
+  Z = __float2int_rn(fminf(fmaxf(__fmul_rn(-lo, inv_s), -1073741824.0f), 1073741824.0f));
+#else
+  volatile float d = hi - lo;
+  volatile float w = d * (1.0f / (float)(1u << bits));
+  s = w > 1e-8f ? (float)w : 1e-8f;
+  volatile float inv = 1.0f / s;
+  inv_s = inv;
+  volatile float t = -lo * inv_s;
+  float tc = t < -1073741824.0f ? -1073741824.0f : (t > 1073741824.0f ? 1073741824.0f : (float)t);
+  Z = (int)__builtin_rintf(tc);
+#endif
+}
+
+#ifdef __CUDACC__
+// Eq. 1: q = min(max(rint(x * inv_s) + Z, 0), L); NaN -> 0 (fmaxf returns the non-NaN operand).
+__device__ __forceinline__ int quantize_code(float x, float inv_s, float Zf, float Lf) {
+  float u = __fadd_rn(rintf(__fmul_rn(x, inv_s)), Zf);
+  return __float2int_rn(fminf(fmaxf(u, 0.0f), Lf));
+}
+
+// ------------------------------------------------------------------ shared-memory addresses
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+// ------------------------------------------------------------------ mbarrier
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded wait: gives up after about a second (2^31 SM clocks) or as soon as another
+// thread of the CTA has raised `*abort_flag`.  Returns false when it gave up; the caller
+// must then leave through the kernel's common exit path.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  uint32_t spins = 0;
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((++spins & 63u) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > (1ll << 31)) {
+        *abort_flag = 1;
+        record_error(DGQ_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void fence_barrier_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// ------------------------------------------------------------------ TMA tile loads (each CTA fetches its own tiles)
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* m) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* m, uint64_t* bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* m, uint64_t* bar, int c0, int c1,
+                                            int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], "
+      "[%2];" ::"r"(smem_u32(dst)),
+      "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+
+// ------------------------------------------------------------------ tcgen05 / tensor memory
+__device__ __forceinline__ void tmem_alloc(uint32_t* smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)),
+               "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+// One 128 x N x 32 int8 MMA: D[tmem] (+)= A[smem] * B[smem]^T, issued by a single thread.
+__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                       uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrives on `bar` once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void mma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+// 32 lanes x 16 consecutive 32-bit columns: thread i of the warp receives row (lane base + i).
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, K-major operand, rows of 128 B (SWIZZLE_128B) or 32 B (SWIZZLE_32B):
+// start address >> 4 in bits [0,14), stride between 8-row groups >> 4 in bits [32,46), descriptor
+// version 1 in bits [46,48), swizzle mode in bits [61,64) (2 = 128 B, 6 = 32 B).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t sbo_bytes, uint32_t layout) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)layout << 61);
+}
+#endif  // __CUDACC__
+
+}  // namespace dgq
