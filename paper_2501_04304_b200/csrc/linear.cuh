@@ -1,0 +1,517 @@
+// Group-quantized layer: int8 tensor-core GEMM (tcgen05.mma kind::i8, accumulators in tensor
+// memory) whose accumulator is switched at every channel-group boundary, with the per-group
+// de-quantizing epilogue
+//     Y[t,o] = bias[o] + sw[o] * sum_g s[t,g] * (acc_g[t,o] - Z[t,g] * wsum_g[o])
+// (Eq. 1's de-quantizer with the group parameters of Eq. 6) fused in.
+//
+// CTA = one 128-row output tile x BN columns, persistent over tiles.  Warp roles:
+//   warps 0-7   epilogue: lane quarter = warp & 3 (the TMEM lanes a warp may read), column half = warp >> 2
+//   warp  8     TMA producer (one elected lane): A code tile and B weight tile per 128-byte K stage
+//   warp  9     MMA issuer (one elected lane) and TMEM allocator
+//   warps 10-13 (4-bit weights only) unpack packed nibbles from global memory into the B stage
+// K runs over 32-code atoms; a stage holds four atoms.  Group segments are multiples of one atom,
+// so the issuer moves to the next TMEM accumulator between two atoms, commits the finished one to
+// the epilogue and keeps going while the epilogue drains it.
+// Linear layers: A and B stages are 128-byte-swizzled tiles fetched with one TMA box each.
+// 3x3 conv (implicit GEMM): the reduction order is group-major, then filter tap, then channel
+// atom; every A atom is its own 32-byte-swizzled 4-D TMA box of the NHWC code tensor shifted by
+// the tap, out-of-image rows zero-filled by TMA (exact for zero-centred codes).
+#pragma once
+
+#include "weights.cuh"
+
+namespace dgq {
+
+constexpr int GEMM_BM = 128;
+constexpr int GEMM_EPI_WARPS = 8;
+constexpr int GEMM_A_STAGE = GEMM_BM * 128;  // bytes
+constexpr int GEMM_SMEM_LIMIT = 227 * 1024;
+
+template <int BN>
+struct GemmCfg {
+  static constexpr int B_STAGE = BN * 128;
+  static constexpr int STAGE = GEMM_A_STAGE + B_STAGE;
+  static constexpr int STAGES_RAW = (GEMM_SMEM_LIMIT - 3072) / STAGE;
+  static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
+  static constexpr int NACC_RAW = 512 / BN;
+  static constexpr int NACC = NACC_RAW > 4 ? 4 : NACC_RAW;
+  static constexpr int CH = BN / 2;  // columns per epilogue thread
+  static constexpr int SMEM = STAGES * STAGE + 2048 + 1024;
+  static_assert(BN % 32 == 0 && BN <= 256, "BN must be a multiple of 32 up to 256");
+  static_assert(NACC >= 2, "need two accumulators to overlap the epilogue");
+  static_assert(NACC * BN <= 512, "tensor memory has 512 columns");
+  static_assert(STAGES >= 3, "pipeline too shallow");
+};
+
+struct GemmArgs {
+  int64_t M;
+  int N, N_pad, Kt, G, P;
+  int n_tiles_m, n_tiles_n;
+  uint32_t idesc;
+  int use_zp;                 // 0 for zero-centred codes
+  int per_token;              // 1: scale rows indexed by token, 0: by row_group[token mod P]
+  const float* scale;         // [rows][G]
+  const int32_t* zp;          // [rows][G]
+  const int32_t* row_group;   // [P]
+  const float* sw;            // [N_pad]
+  const float* wsum;          // [G][N_pad]
+  const __half* bias;         // [N] or null
+  __half* Y;
+  int64_t ldy;
+  const uint8_t* w_packed;    // 4-bit weights [N_pad][Kt/2]
+  int seg_end[DGQ_MAX_GROUPS];    // end atom of every group segment
+  // conv
+  int conv_W, conv_H, box_w, box_h, box_n;
+  int grp_atoms[DGQ_MAX_GROUPS];  // channel atoms of every group
+  int grp_chan0[DGQ_MAX_GROUPS];  // first padded channel position of every group
+};
+
+struct __align__(8) GemmShared {
+  uint64_t full[8];
+  uint64_t empty[8];
+  uint64_t acc_full[4];
+  uint64_t acc_empty[4];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+template <int BN, bool W4, bool CONV>
+__global__ void __launch_bounds__(W4 ? 448 : 320, 1)
+gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ GemmArgs a) {
+  using Cfg = GemmCfg<BN>;
+  constexpr int STAGES = Cfg::STAGES;
+  constexpr int NACC = Cfg::NACC;
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) &
+                                                         ~uintptr_t(1023));
+  unsigned char* smA = smem;
+  unsigned char* smB = smem + STAGES * GEMM_A_STAGE;
+  GemmShared* sh = reinterpret_cast<GemmShared*>(smem + STAGES * Cfg::STAGE);
+  volatile int* abort_flag = &sh->abort_flag;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int n_atoms = a.Kt >> 5;
+  const int n_kstages = (n_atoms + 3) >> 2;
+  const int n_tiles = a.n_tiles_m * a.n_tiles_n;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < STAGES; ++i) {
+      mbar_init(&sh->full[i], W4 ? 5 : 1);
+      mbar_init(&sh->empty[i], 1);
+    }
+    for (int i = 0; i < NACC; ++i) {
+      mbar_init(&sh->acc_full[i], 1);
+      mbar_init(&sh->acc_empty[i], GEMM_EPI_WARPS);
+    }
+    sh->abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 9) {
+    tmem_alloc(&sh->tmem_base, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = sh->tmem_base;
+
+  if (warp == 8) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      tma_prefetch_desc(&tmA);
+      if (!W4) tma_prefetch_desc(&tmB);
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const int tm = tile / a.n_tiles_n, tn = tile - tm * a.n_tiles_n;
+        const int m0 = tm * GEMM_BM, n0 = tn * BN;
+        int cw = 0, chh = 0, cn = 0;  // conv: spatial origin of this row tile
+        if (CONV) {
+          const int hw = a.conv_H * a.conv_W;
+          cn = m0 / hw;
+          const int rem = m0 - cn * hw;
+          chh = rem / a.conv_W;
+          cw = rem - chh * a.conv_W;
+        }
+        int g = 0, g_start = 0;  // conv: current group and its first atom
+        for (int ks = 0; ks < n_kstages && ok; ++ks, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          ok = mbar_wait(&sh->empty[s], ph ^ 1, abort_flag);
+          if (!ok) break;
+          const int atoms_here = min(4, n_atoms - ks * 4);
+          uint32_t bytes = W4 ? 0u : (uint32_t)Cfg::B_STAGE;
+          bytes += CONV ? (uint32_t)(atoms_here * 4096) : (uint32_t)GEMM_A_STAGE;
+          mbar_arrive_expect_tx(&sh->full[s], bytes);
+          if (CONV) {
+            for (int j = 0; j < atoms_here; ++j) {
+              const int atom = ks * 4 + j;
+              while (atom >= a.seg_end[g]) {
+                g_start = a.seg_end[g];
+                ++g;
+              }
+              const int local = atom - g_start;
+              const int tap = local / a.grp_atoms[g];
+              const int ca = local - tap * a.grp_atoms[g];
+              const int ky = tap / 3, kx = tap - ky * 3;
+              tma_load_4d(smA + s * GEMM_A_STAGE + j * 4096, &tmA, &sh->full[s], a.grp_chan0[g] + ca * 32,
+                          cw + kx - 1, chh + ky - 1, cn);
+            }
+          } else {
+            tma_load_2d(smA + s * GEMM_A_STAGE, &tmA, &sh->full[s], ks * 128, m0);
+          }
+          if (!W4) tma_load_2d(smB + s * Cfg::B_STAGE, &tmB, &sh->full[s], ks * 128, n0);
+        }
+      }
+    }
+  } else if (warp == 9) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t it = 0, acc_it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        int g = 0;
+        bool first = true;
+        int ab = acc_it % NACC;
+        ok = mbar_wait(&sh->acc_empty[ab], ((acc_it / NACC) & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        for (int ks = 0; ks < n_kstages && ok; ++ks, ++it) {
+          const int s = it % STAGES;
+          ok = mbar_wait(&sh->full[s], (it / STAGES) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const int atoms_here = min(4, n_atoms - ks * 4);
+          const uint32_t a_addr = smem_u32(smA + s * GEMM_A_STAGE);
+          const uint32_t b_addr = smem_u32(smB + s * Cfg::B_STAGE);
+          for (int j = 0; j < atoms_here && ok; ++j) {
+            const int atom = ks * 4 + j;
+            if (atom >= a.seg_end[g]) {  // group finished: hand its accumulator to the epilogue
+              mma_commit(&sh->acc_full[ab]);
+              ++acc_it;
+              ++g;
+              first = true;
+              ab = acc_it % NACC;
+              ok = mbar_wait(&sh->acc_empty[ab], ((acc_it / NACC) & 1) ^ 1, abort_flag);
+              if (!ok) break;
+              tc_fence_after();
+            }
+            const uint64_t da = CONV ? smem_desc(a_addr + j * 4096, 256, 6) : smem_desc(a_addr + j * 32, 1024, 2);
+            const uint64_t db = smem_desc(b_addr + j * 32, 1024, 2);
+            mma_i8(tmem_base + (uint32_t)(ab * BN), da, db, a.idesc, first ? 0u : 1u);
+            first = false;
+          }
+          if (ok) mma_commit(&sh->empty[s]);  // stage reusable once these MMAs have read it
+        }
+        if (ok) {
+          mma_commit(&sh->acc_full[ab]);
+          ++acc_it;
+        }
+      }
+    }
+  } else if (warp < GEMM_EPI_WARPS) {
+    // ------------------------------------------------------------ epilogue
+    constexpr int CH = Cfg::CH;
+    const int q = warp & 3, half = warp >> 2;
+    uint32_t acc_it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      const int tm = tile / a.n_tiles_n, tn = tile - tm * a.n_tiles_n;
+      const int64_t row = (int64_t)tm * GEMM_BM + q * 32 + lane;
+      const int64_t row_c = row < a.M ? row : a.M - 1;
+      const int col0 = tn * BN + half * CH;
+      const int64_t prow = a.per_token ? row_c : (int64_t)a.row_group[row_c % a.P];
+      const float* srow = a.scale + prow * a.G;
+      const int32_t* zrow = a.zp + prow * a.G;
+      float y[CH];
+#pragma unroll
+      for (int i = 0; i < CH; ++i) y[i] = 0.f;
+      for (int g = 0; g < a.G && ok; ++g, ++acc_it) {
+        const float s = __ldg(srow + g);
+        const float c = a.use_zp ? -s * (float)__ldg(zrow + g) : 0.f;
+        const int ab = acc_it % NACC;
+        ok = __all_sync(0xffffffffu, mbar_wait(&sh->acc_full[ab], (acc_it / NACC) & 1, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * BN + half * CH);
+        const float* ws = a.wsum + (size_t)g * a.N_pad + col0;
+#pragma unroll
+        for (int cc = 0; cc < CH; cc += 16) {
+          uint32_t r[16];
+          tmem_ld16(taddr + cc, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) y[cc + i] = fmaf(s, (float)(int)r[i], y[cc + i]);
+          if (a.use_zp) {
+#pragma unroll
+            for (int i = 0; i < 16; i += 4) {
+              const float4 w4 = __ldg(reinterpret_cast<const float4*>(ws + cc + i));
+              y[cc + i] = fmaf(c, w4.x, y[cc + i]);
+              y[cc + i + 1] = fmaf(c, w4.y, y[cc + i + 1]);
+              y[cc + i + 2] = fmaf(c, w4.z, y[cc + i + 2]);
+              y[cc + i + 3] = fmaf(c, w4.w, y[cc + i + 3]);
+            }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh->acc_empty[ab]);
+      }
+      if (!ok) break;
+      if (row < a.M) {
+        __half* yrow = a.Y + row * a.ldy;
+#pragma unroll
+        for (int i = 0; i < CH; i += 8) {
+          const int col = col0 + i;
+          if (col < a.N) {
+            const float4 s0 = __ldg(reinterpret_cast<const float4*>(a.sw + col));
+            const float4 s1 = __ldg(reinterpret_cast<const float4*>(a.sw + col + 4));
+            float b[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            if (a.bias) {
+              const uint4 bv = __ldg(reinterpret_cast<const uint4*>(a.bias + col));
+              const __half2* bh = reinterpret_cast<const __half2*>(&bv);
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const float2 f = __half22float2(bh[k]);
+                b[2 * k] = f.x;
+                b[2 * k + 1] = f.y;
+              }
+            }
+            const float sw8[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+            uint4 o;
+            __half2* oh = reinterpret_cast<__half2*>(&o);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              oh[k] = __floats2half2_rn(fmaf(sw8[2 * k], y[i + 2 * k], b[2 * k]),
+                                        fmaf(sw8[2 * k + 1], y[i + 2 * k + 1], b[2 * k + 1]));
+            *reinterpret_cast<uint4*>(yrow + col) = o;
+          }
+        }
+      }
+    }
+  } else if (W4) {
+    // ------------------------------------------------------------ 4-bit weight unpack into the B stage
+    const int ut = threadIdx.x - 320;  // 0..127
+    uint32_t it = 0;
+    bool ok = true;
+    const int row_bytes = a.Kt >> 1;
+    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      const int tn = tile % a.n_tiles_n;
+      const int n0 = tn * BN;
+      for (int ks = 0; ks < n_kstages && ok; ++ks, ++it) {
+        const int s = it % STAGES;
+        ok = __all_sync(0xffffffffu, mbar_wait(&sh->empty[s], ((it / STAGES) & 1) ^ 1, abort_flag));
+        if (!ok) break;
+        unsigned char* bst = smB + s * Cfg::B_STAGE;
+        for (int item = ut; item < BN * 4; item += 128) {
+          const int r = item >> 2, qd = item & 3;  // B row, 16-byte packed quarter of the 64-byte row slice
+          const int kb = ks * 64 + qd * 16;
+          uint4 pk = make_uint4(0u, 0u, 0u, 0u);
+          if (kb < row_bytes)
+            pk = __ldg(reinterpret_cast<const uint4*>(a.w_packed + (size_t)(n0 + r) * row_bytes + kb));
+          const uint4 c0 = make_uint4((pk.x << 4) & 0xF0F0F0F0u, pk.x & 0xF0F0F0F0u, (pk.y << 4) & 0xF0F0F0F0u,
+                                      pk.y & 0xF0F0F0F0u);
+          const uint4 c1 = make_uint4((pk.z << 4) & 0xF0F0F0F0u, pk.z & 0xF0F0F0F0u, (pk.w << 4) & 0xF0F0F0F0u,
+                                      pk.w & 0xF0F0F0F0u);
+          // 128-byte swizzle: 16-byte chunk index XOR (row mod 8) inside every 8-row, 1024-byte group
+          unsigned char* rowp = bst + (r >> 3) * 1024 + (r & 7) * 128;
+          *reinterpret_cast<uint4*>(rowp + (((2 * qd) ^ (r & 7)) << 4)) = c0;
+          *reinterpret_cast<uint4*>(rowp + (((2 * qd + 1) ^ (r & 7)) << 4)) = c1;
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh->full[s]);
+      }
+    }
+  }
+
+  // ------------------------------------------------------------ common exit
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    // give copies that may still be in flight time to land before the CTA's shared memory is released
+    const long long t0 = clock64();
+    while (clock64() - t0 < 200000) {
+    }
+    __syncthreads();
+  }
+  if (warp == 9) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+static bool encode_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides,
+                       const uint32_t* box, CUtensorMapSwizzle sw) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint64_t d[5];
+  cuuint64_t st[5];
+  cuuint32_t b[5], es[5];
+  for (int i = 0; i < rank; ++i) {
+    d[i] = dims[i];
+    b[i] = box[i];
+    es[i] = 1;
+  }
+  for (int i = 0; i + 1 < rank; ++i) st[i] = strides[i];
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void*>(base), d, st, b, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN, bool W4, bool CONV>
+static dgq_status launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& a, int grid,
+                              cudaStream_t stream) {
+  using Cfg = GemmCfg<BN>;
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  DGQ_CUDA_OK(cudaGetDevice(&dev));
+  if (dev >= 64 || !attr_set[dev]) {
+    DGQ_CUDA_OK(cudaFuncSetAttribute(gq_gemm_kernel<BN, W4, CONV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     Cfg::SMEM));
+    if (dev < 64) attr_set[dev] = true;
+  }
+  gq_gemm_kernel<BN, W4, CONV><<<grid, W4 ? 448 : 320, Cfg::SMEM, stream>>>(tmA, tmB, a);
+  g_launches += 1;
+  DGQ_CUDA_OK(cudaGetLastError());
+  return DGQ_OK;
+}
+
+template <int BN>
+static dgq_status launch_gemm_bn(bool w4, bool conv, const CUtensorMap& tmA, const CUtensorMap& tmB,
+                                 const GemmArgs& a, int grid, cudaStream_t stream) {
+  if (w4)
+    return conv ? launch_gemm<BN, true, true>(tmA, tmB, a, grid, stream)
+                : launch_gemm<BN, true, false>(tmA, tmB, a, grid, stream);
+  return conv ? launch_gemm<BN, false, true>(tmA, tmB, a, grid, stream)
+              : launch_gemm<BN, false, false>(tmA, tmB, a, grid, stream);
+}
+
+}  // namespace dgq
+
+extern "C" dgq_status dgq_linear(const dgq_groups* g, const dgq_weight* w, int timestep, int mode, int layout,
+                                 const void* Xq, const float* dyn_scale, const int32_t* dyn_zp, const void* bias,
+                                 void* Y, int64_t M, int64_t ldy, const dgq_conv_desc* conv, void* stream) {
+  using namespace dgq;
+  if (!g || !w || !Xq || !Y || M <= 0) return DGQ_ERR_INVALID_ARG;
+  if (mode != DGQ_MODE_STATIC && mode != DGQ_MODE_DYNAMIC_TOKEN) return DGQ_ERR_INVALID_ARG;
+  if (layout != DGQ_CODES_U8 && layout != DGQ_CODES_S8_CENTRED) return DGQ_ERR_INVALID_ARG;
+  if (timestep < 0 || timestep >= g->T) return DGQ_ERR_INVALID_ARG;
+  if (w->C != g->C || w->G != g->G || ldy < w->N) return DGQ_ERR_INVALID_ARG;
+  if ((conv != nullptr) != (w->is_conv != 0)) return DGQ_ERR_INVALID_ARG;
+  if (!aligned16(Xq) || !aligned16(Y) || (ldy % 8) != 0 || (bias && !aligned16(bias))) return DGQ_ERR_ALIGNMENT;
+  if (M > (int64_t)INT32_MAX - 256) return DGQ_ERR_UNSUPPORTED;
+  GemmArgs a;
+  std::memset(&a, 0, sizeof(a));
+  if (mode == DGQ_MODE_STATIC) {
+    if (!g->filled[timestep]) return DGQ_ERR_NOT_CALIBRATED;
+    const size_t trow = (size_t)timestep * g->R * g->G;
+    a.scale = g->d_scale + trow;
+    a.zp = g->d_zp + trow;
+    a.per_token = 0;
+  } else {
+    if (!dyn_scale || !dyn_zp) return DGQ_ERR_INVALID_ARG;
+    if (layout != DGQ_CODES_U8) return DGQ_ERR_UNSUPPORTED;
+    a.scale = dyn_scale;
+    a.zp = dyn_zp;
+    a.per_token = 1;
+  }
+  a.M = M;
+  a.N = w->N;
+  a.N_pad = w->N_pad;
+  a.Kt = w->Kt;
+  a.G = g->G;
+  a.P = g->P;
+  a.use_zp = (layout == DGQ_CODES_U8);
+  a.row_group = g->d_row_group;
+  a.sw = w->d_sw;
+  a.wsum = w->d_wsum;
+  a.bias = (const __half*)bias;
+  a.Y = (__half*)Y;
+  a.ldy = ldy;
+  a.w_packed = (const uint8_t*)w->d_w;
+  for (int k = 0; k < g->G; ++k) {
+    a.seg_end[k] = w->seg_end[k];
+    a.grp_atoms[k] = (g->group_off[k + 1] - g->group_off[k]) / DGQ_K_ATOM;
+    a.grp_chan0[k] = g->group_off[k];
+  }
+  int BN = 128;
+  if (w->N % 160 == 0) BN = 160;
+  else if (w->N <= 64) BN = 64;
+  // instruction descriptor of kind::i8: int32 accumulator (bits 4-5 = 2), A format bit 7 (0 = u8,
+  // 1 = s8), B format bit 10 = 1 (s8), both K-major, N >> 3 at bit 17, M >> 4 at bit 24
+  a.idesc = (2u << 4) | ((layout == DGQ_CODES_S8_CENTRED ? 1u : 0u) << 7) | (1u << 10) |
+            ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(GEMM_BM >> 4) << 24);
+  a.n_tiles_m = (int)((M + GEMM_BM - 1) / GEMM_BM);
+  a.n_tiles_n = (w->N + BN - 1) / BN;
+
+  CUtensorMap tmA, tmB;
+  std::memset(&tmA, 0, sizeof(tmA));
+  std::memset(&tmB, 0, sizeof(tmB));
+  if (conv) {
+    if (layout != DGQ_CODES_S8_CENTRED || mode != DGQ_MODE_STATIC || g->R != 1) return DGQ_ERR_UNSUPPORTED;
+    if (conv->c != g->C || (int64_t)conv->n * conv->h * conv->w != M) return DGQ_ERR_INVALID_ARG;
+    int bw, bh, bn;
+    if (conv->w >= 128) {
+      if (conv->w % 128) return DGQ_ERR_UNSUPPORTED;
+      bw = 128, bh = 1, bn = 1;
+    } else if (128 % conv->w) {
+      return DGQ_ERR_UNSUPPORTED;
+    } else if (conv->h * conv->w >= 128) {
+      bw = conv->w, bh = 128 / conv->w, bn = 1;
+      if (conv->h % bh) return DGQ_ERR_UNSUPPORTED;
+    } else {
+      if (128 % (conv->h * conv->w)) return DGQ_ERR_UNSUPPORTED;
+      bw = conv->w, bh = conv->h, bn = 128 / (conv->h * conv->w);
+    }
+    a.conv_W = conv->w;
+    a.conv_H = conv->h;
+    a.box_w = bw;
+    a.box_h = bh;
+    a.box_n = bn;
+    const uint64_t Cp = (uint64_t)g->K_pad;
+    const uint64_t dims[4] = {Cp, (uint64_t)conv->w, (uint64_t)conv->h, (uint64_t)conv->n};
+    const uint64_t strides[3] = {Cp, Cp * conv->w, Cp * conv->w * conv->h};
+    const uint32_t box[4] = {32u, (uint32_t)bw, (uint32_t)bh, (uint32_t)bn};
+    if (!encode_map(&tmA, Xq, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_32B)) return DGQ_ERR_CUDA;
+  } else {
+    const uint64_t dims[2] = {(uint64_t)g->K_pad, (uint64_t)M};
+    const uint64_t strides[1] = {(uint64_t)g->K_pad};
+    const uint32_t box[2] = {128u, (uint32_t)GEMM_BM};
+    if (!encode_map(&tmA, Xq, 2, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) return DGQ_ERR_CUDA;
+  }
+  if (w->w_bits == 8) {
+    const uint64_t dims[2] = {(uint64_t)w->Kt, (uint64_t)w->N_pad};
+    const uint64_t strides[1] = {(uint64_t)w->Kt};
+    const uint32_t box[2] = {128u, (uint32_t)BN};
+    if (!encode_map(&tmB, w->d_w, 2, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) return DGQ_ERR_CUDA;
+  }
+  int dev = 0, n_sm = 148;
+  DGQ_CUDA_OK(cudaGetDevice(&dev));
+  DGQ_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+  const int grid = std::min(a.n_tiles_m * a.n_tiles_n, n_sm);
+  const bool w4 = (w->w_bits == 4);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (BN == 160) return launch_gemm_bn<160>(w4, conv != nullptr, tmA, tmB, a, grid, st);
+  if (BN == 64) return launch_gemm_bn<64>(w4, conv != nullptr, tmA, tmB, a, grid, st);
+  return launch_gemm_bn<128>(w4, conv != nullptr, tmA, tmB, a, grid, st);
+}

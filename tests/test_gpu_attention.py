@@ -1,0 +1,84 @@
+"""GPU parity: cross-attention with log2-quantized scores against the fp64 oracle."""
+import numpy as np
+import pytest
+
+from oracle import attention as oa
+from paper_2501_04304_b200 import synth
+from dgq_testlib import gpu, to_dev, check_output
+
+pytestmark = pytest.mark.gpu
+
+
+def _compare(torch, b, Q, K, V, bits, gran=0, fixed=None, code_frac=1e-4, out_rel=1e-3):
+    O_ref, codes_ref, s_ref, A = oa.cross_attn_logq(Q, K, V, bits, gran, fixed)
+    fx = to_dev(torch, np.asarray(fixed, np.float32)) if fixed is not None else None
+    O, scale, codes = b.cross_attn_logq(to_dev(torch, Q), to_dev(torch, K), to_dev(torch, V), bits, gran, fx,
+                                        want_scale=True, want_codes=True)
+    assert b.device_status() == 0
+    s_gpu = scale.cpu().numpy().astype(np.float64)
+    assert np.allclose(s_gpu, s_ref.ravel(), rtol=2e-5, atol=0)
+    c = codes.cpu().numpy().astype(np.int64)
+    diff = np.abs(c - codes_ref)
+    assert diff.max() <= 1, "a code differs by more than one level"
+    frac = (diff != 0).mean()
+    assert frac <= code_frac, f"{frac:.2e} of the codes differ"
+    check_output(O, O_ref, out_rel)
+    return frac
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_small_config3_like(bits):
+    torch, b = gpu()
+    Q, K, V = synth.attention_inputs(3, 2, 8, 300, 77, 40)
+    _compare(torch, b, Q, K, V, bits)
+
+
+@pytest.mark.parametrize("B,H,nq,nk,d", [
+    (1, 1, 16, 3, 40),       # tiny: one warp slab, nk far below the padded width
+    (2, 3, 130, 77, 80),     # ragged row block
+    (1, 2, 64, 77, 160),
+    (1, 2, 257, 100, 64),    # nk > 80 path
+    (2, 2, 40, 128, 128),
+    (3, 1, 129, 2, 40),      # smallest legal nk
+])
+def test_shapes(B, H, nq, nk, d):
+    torch, b = gpu()
+    Q, K, V = synth.attention_inputs(4, B, H, nq, nk, d, ctx_dim=64)
+    _compare(torch, b, Q, K, V, 8, code_frac=5e-4)
+
+
+@pytest.mark.parametrize("gran", [0, 1, 2])
+def test_scale_granularity(gran):
+    torch, b = gpu()
+    Q, K, V = synth.attention_inputs(5, 3, 4, 200, 77, 40, ctx_dim=64)
+    _compare(torch, b, Q, K, V, 6, gran=gran, code_frac=5e-4)
+
+
+def test_fixed_scale_variant():
+    torch, b = gpu()
+    Q, K, V = synth.attention_inputs(6, 2, 2, 128, 77, 40, ctx_dim=64)
+    _compare(torch, b, Q, K, V, 8, fixed=[0.05, 0.01], code_frac=5e-4)
+
+
+def test_wide_logits_saturate_four_bits():
+    """Spread-out logits: 4-bit codes clamp at 15 and the 8-bit codes run far past the fp16 range."""
+    torch, b = gpu()
+    Q, K, V = synth.attention_inputs(7, 1, 2, 256, 77, 40, ctx_dim=64)
+    K = (K.astype(np.float32) * 6).astype(np.float16)
+    K[:, 0, :, -1] = np.float16(6.0 * np.sqrt(40))
+    for bits in (4, 8):
+        O_ref, codes_ref, _, _ = oa.cross_attn_logq(Q, K, V, bits)
+        assert codes_ref.max() == (15 if bits == 4 else codes_ref.max()) and codes_ref.max() >= 15
+        _compare(torch, b, Q, K, V, bits, code_frac=1e-3)
+
+
+def test_argument_errors():
+    torch, b = gpu()
+    Q, K, V = synth.attention_inputs(8, 1, 1, 16, 4, 40, ctx_dim=16)
+    Qd, Kd, Vd = to_dev(torch, Q), to_dev(torch, K), to_dev(torch, V)
+    with pytest.raises(b.DgqError) as e:
+        b.cross_attn_logq(Qd, Kd[:, :1].contiguous(), Vd[:, :1].contiguous())
+    assert e.value.status == 1
+    with pytest.raises(b.DgqError) as e:
+        b.cross_attn_logq(Qd, Kd, Vd, workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 4
