@@ -1,0 +1,411 @@
+#!/usr/bin/env python
+"""Benchmark of the DGQ hot path on one B200 (or N independent replicas, one per rank).
+
+One step = one pass of the whole path over one batch of synthetic, seeded tensors shaped like
+the 64x64-latent level of the Stable Diffusion v1.4 UNet at batch 2 (classifier-free guidance):
+
+  * transformer-block linears, W8A8, per-token dynamic activation scales over 8 calibrated
+    channel groups: activation quantizer + proj_in, q/k/v (one quantizer call feeds three
+    GEMMs), out (320 -> 320), GEGLU FF 320 -> 2560 and 1280 -> 320, 8192 tokens;
+  * cross-attention with prompt-specific log2 score quantization, B = 2, 8 heads,
+    4096 queries x 40, 77 keys, 8-bit scores;
+  * the level's ResBlock 3x3 convolution, 320 -> 320 on 2 x 64 x 64, W4A6, 16 channel groups,
+    as an implicit GEMM (activation quantizer + conv).
+
+Calibration and weight preparation are offline and untimed.  Buffers rotate over enough
+distinct sets that the footprint exceeds L2, so the timed kernels read HBM.
+
+`value` is the algorithmic int8 throughput of the whole step (2 M N K_real of every GEMM and
+conv, divided by the full step time including quantizers and attention).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2501_04304_b200 import synth  # noqa: E402
+
+SEED = 1
+TOKENS, BATCH = 4096, 2
+M = TOKENS * BATCH
+LINEARS = [  # name, N, K, input id
+    ("proj_in", 320, 320, "a"), ("q", 320, 320, "b"), ("k", 320, 320, "b"), ("v", 320, 320, "b"),
+    ("out", 320, 320, "c"), ("ff1", 2560, 320, "d"), ("ff2", 320, 1280, "e"),
+]
+INPUT_C = {"a": 320, "b": 320, "c": 320, "d": 320, "e": 1280}
+ATT = dict(B=2, H=8, nq=4096, nk=77, d=40, bits=8)
+CONV = dict(n=2, h=64, w=64, c=320, N=320)
+WORKLOAD = ("sdv14_64x64_level_batch2: W8A8 transformer linears (proj_in,q,k,v,out 320->320, FF 320->2560, "
+            "1280->320; 8192 tokens; dynamic per-token scales, 8 channel groups) + log2 cross-attention "
+            "(B2 H8 nq4096 d40 nk77, 8-bit) + W4A6 3x3 conv 320->320 on 2x64x64 (16 groups)")
+
+
+def gemm_ops():
+    ops = sum(2.0 * M * N * K for _, N, K, _ in LINEARS)
+    ops += 2.0 * CONV["n"] * CONV["h"] * CONV["w"] * CONV["N"] * 9 * CONV["c"]
+    return ops
+
+
+def attn_bytes():
+    a = ATT
+    return 2.0 * a["B"] * a["nq"] * a["H"] * a["d"] * 2 + 2.0 * a["B"] * a["nk"] * a["H"] * a["d"] * 2
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm=float(d["hbm_gbs"]), bf16=float(d["bf16_tflops"]),
+                    bf16_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler(threading.Thread):
+    """Samples nvidia-smi SM clocks and throttle reasons while the timed region runs."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self._stop_evt = threading.Event()
+
+    def run(self):
+        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        while not self._stop_evt.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-i",
+                                      str(self.index)], capture_output=True, text=True, timeout=5).stdout
+                f = [x.strip() for x in out.strip().split(",")]
+                self.samples.append(float(f[0]))
+                self.max_mhz = float(f[1])
+                for n, v in zip(names, f[2:]):
+                    if v.lower().startswith("active"):
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            self._stop_evt.wait(0.1)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=10)
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------------------ CUDA arm
+class Workload:
+    """Calibrated layers, prepared weights and rotating buffer sets on one GPU."""
+
+    def __init__(self, torch, b, n_sets):
+        self.torch, self.b, self.n_sets = torch, b, n_sets
+        dev = "cuda"
+        self.groups, self.weights, self.biases = {}, {}, {}
+        # one grouping per distinct layer input; calibrated on 4 further draws
+        for key, C in INPUT_C.items():
+            Xcal = torch.from_numpy(synth.activations(SEED, 100 + ord(key), 4, TOKENS, C)).to(dev)
+            self.groups[key] = b.calibrate_groups(Xcal, TOKENS, 8, 8, b.DIM_CHANNEL)
+            del Xcal
+        for i, (name, N, K, key) in enumerate(LINEARS):
+            W = torch.from_numpy(synth.weights(SEED, 200 + i, N, K)).to(dev)
+            self.weights[name] = b.weight_prepare(self.groups[key], W, 8)
+            self.biases[name] = torch.from_numpy(synth.bias(SEED, 300 + i, N)).to(dev)
+        c = CONV
+        Xcal = torch.from_numpy(synth.activations(SEED, 150, 4, c["h"] * c["w"], c["c"], token_outliers=False)).to(dev)
+        self.conv_groups = b.calibrate_groups(Xcal, c["h"] * c["w"], 6, 16, b.DIM_CHANNEL)
+        del Xcal
+        self.conv_desc = (c["n"], c["h"], c["w"], c["c"])
+        Wc = torch.from_numpy(synth.conv_weights(SEED, 250, c["N"], c["c"])).to(dev)
+        self.conv_weight = b.weight_prepare(self.conv_groups, Wc, 4, conv=self.conv_desc)
+        self.conv_bias = torch.from_numpy(synth.bias(SEED, 350, c["N"])).to(dev)
+        # host inputs (pinned) and device buffer sets
+        self.host = {}
+        for key, C in INPUT_C.items():
+            self.host[key] = torch.from_numpy(synth.activations(SEED, 10 + ord(key), BATCH, TOKENS, C)).pin_memory()
+        self.host["conv"] = torch.from_numpy(
+            synth.activations(SEED, 60, c["n"], c["h"] * c["w"], c["c"], token_outliers=False)).pin_memory()
+        a = ATT
+        Q, K, V = synth.attention_inputs(SEED, a["B"], a["H"], a["nq"], a["nk"], a["d"])
+        self.host["Q"], self.host["K"], self.host["V"] = [torch.from_numpy(x).pin_memory() for x in (Q, K, V)]
+        ws_bytes = b.cross_attn_workspace_bytes(a["B"], a["H"], a["nq"], a["nk"], a["d"])
+        self.sets = []
+        for _ in range(n_sets):
+            s = {"in": {k: v.to(dev) for k, v in self.host.items()}}
+            s["codes"], s["ds"], s["dz"] = {}, {}, {}
+            for key in INPUT_C:
+                g = self.groups[key]
+                s["codes"][key] = torch.empty((M, g.K_pad), dtype=torch.uint8, device=dev)
+                s["ds"][key] = torch.empty((M, g.G), dtype=torch.float32, device=dev)
+                s["dz"][key] = torch.empty((M, g.G), dtype=torch.int32, device=dev)
+            s["conv_codes"] = torch.empty((M, self.conv_groups.K_pad), dtype=torch.uint8, device=dev)
+            s["out"] = {name: torch.empty((M, N), dtype=torch.float16, device=dev) for name, N, _, _ in LINEARS}
+            s["conv_out"] = torch.empty((M, c["N"]), dtype=torch.float16, device=dev)
+            s["attn_out"] = torch.empty((a["B"], a["nq"], a["H"], a["d"]), dtype=torch.float16, device=dev)
+            s["attn_ws"] = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+            self.sets.append(s)
+        self.host_out = {k: torch.empty((M, 320), dtype=torch.float16).pin_memory() for k in ("ff2", "conv")}
+        self.host_out["attn"] = torch.empty((a["B"], a["nq"], a["H"], a["d"]), dtype=torch.float16).pin_memory()
+
+    def set_bytes(self):
+        tot = 0
+        s = self.sets[0]
+        for v in list(s["in"].values()) + list(s["codes"].values()) + list(s["out"].values()) + \
+                [s["conv_codes"], s["conv_out"], s["attn_out"]]:
+            tot += v.numel() * v.element_size()
+        return tot
+
+    def step(self, i, timers=None):
+        """All kernels of one step on buffer set i.  `timers` collects (kind, start, stop) CUDA events."""
+        b, torch = self.b, self.torch
+        s = self.sets[i % self.n_sets]
+
+        def timed(kind, fn):
+            if timers is None:
+                fn()
+                return
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            timers.append((kind, e0, e1))
+
+        for key in INPUT_C:
+            timed("quantize", lambda key=key: b.quantize_act_into(
+                self.groups[key], s["in"][key], s["codes"][key], s["ds"][key], s["dz"][key],
+                mode=b.MODE_DYNAMIC_TOKEN))
+        for name, N, K, key in LINEARS:
+            timed("gemm", lambda name=name, key=key: b.linear(
+                self.groups[key], self.weights[name], s["codes"][key], mode=b.MODE_DYNAMIC_TOKEN,
+                dyn_scale=s["ds"][key], dyn_zp=s["dz"][key], bias=self.biases[name], out=s["out"][name]))
+        timed("attention", lambda: b.cross_attn_logq(s["in"]["Q"], s["in"]["K"], s["in"]["V"], ATT["bits"],
+                                                     out=s["attn_out"], workspace=s["attn_ws"]))
+        timed("quantize", lambda: b.quantize_act_into(self.conv_groups, s["in"]["conv"], s["conv_codes"], None, None,
+                                                      layout=b.CODES_S8_CENTRED))
+        timed("gemm", lambda: b.linear(self.conv_groups, self.conv_weight, s["conv_codes"],
+                                       layout=b.CODES_S8_CENTRED, bias=self.conv_bias, out=s["conv_out"],
+                                       conv=self.conv_desc))
+
+    def step_e2e(self, i):
+        """The same step through host buffers: inputs copied from pinned memory, results read back."""
+        s = self.sets[i % self.n_sets]
+        for k, h in self.host.items():
+            s["in"][k].copy_(h, non_blocking=True)
+        self.step(i)
+        self.host_out["ff2"].copy_(s["out"]["ff2"], non_blocking=True)
+        self.host_out["conv"].copy_(s["conv_out"], non_blocking=True)
+        self.host_out["attn"].copy_(s["attn_out"], non_blocking=True)
+
+    def h2d_bytes(self):
+        return int(sum(h.numel() * h.element_size() for h in self.host.values()))
+
+    def d2h_bytes(self):
+        return int(sum(h.numel() * h.element_size() for h in self.host_out.values()))
+
+
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2501_04304_b200 import binding as b
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    b.lib()  # fails loudly if the extension is missing
+
+    n_sets = 3
+    wl = Workload(torch, b, n_sets)
+    l2_bytes = torch.cuda.get_device_properties(local).L2_cache_size
+    assert wl.set_bytes() * n_sets > 2 * l2_bytes
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        wl.step(i)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    timers = []
+    launches0 = b.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for i in range(args.steps):
+        wl.step(i, timers)
+    e1.record()
+    barrier()
+    launches = b.launch_count() - launches0
+    ms_total = e0.elapsed_time(e1)
+    # end to end: host buffers in, results out, every step
+    for i in range(2):
+        wl.step_e2e(i)
+    barrier()
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2.record()
+    for i in range(args.steps):
+        wl.step_e2e(i)
+    e3.record()
+    barrier()
+    ms_e2e = e2.elapsed_time(e3)
+    clocks = sampler.stop()
+    status = b.device_status()
+    if status != 0:
+        raise RuntimeError(f"a kernel recorded status {status} ({b.status_string(status)})")
+
+    kind_ms = {}
+    for kind, a0, a1 in timers:
+        kind_ms.setdefault(kind, []).append(a0.elapsed_time(a1))
+    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_step = ms_total / args.steps
+    ops = gemm_ops()
+    value = world * ops / (ms_step * 1e-3) / 1e12
+    e2e_value = world * ops / (ms_e2e / args.steps * 1e-3) / 1e12
+    peaks = measured_peaks()
+    int8_peak = 2.0 * peaks["bf16_sustained"]          # int8 : bf16 dense nominal ratio 4.5 : 2.25
+    gemm_ms = sum(kind_ms["gemm"]) / args.steps        # all GEMM launches of one step
+    gemm_tops = ops / (gemm_ms * 1e-3) / 1e12
+    attn_ms = sum(kind_ms["attention"]) / args.steps
+    quant_ms = sum(kind_ms["quantize"]) / args.steps
+    quant_bytes = 3.0 * (M * sum(INPUT_C.values()) + M * CONV["c"])
+    out = {
+        "metric": "group-quant GEMM TOPS & %INT8 peak; log-quant cross-attn GB/s & %HBM",
+        "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int8", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "l2": f"{n_sets} rotating buffer sets, {wl.set_bytes() * n_sets >> 20} MiB "
+                   f"> L2 {l2_bytes >> 20} MiB", "parallelism": "replicas only" if world > 1 else "single gpu"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "TOPS", "h2d_bytes_per_step": wl.h2d_bytes(),
+                "d2h_bytes_per_step": wl.d2h_bytes(), "ms_per_step": ms_e2e / args.steps},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "achieved": gemm_tops, "peak": int8_peak, "unit": "TOP/s",
+                     "frac": gemm_tops / int8_peak, "traffic": None,
+                     "kernel": "gq_gemm_kernel (8 launches per step)",
+                     "peak_source": f"2 x bf16 sustained, {peaks['source']}"},
+        "kernels": {
+            "gemm": {"ms_per_step": gemm_ms, "tops": gemm_tops, "frac_int8_peak": gemm_tops / int8_peak},
+            "attention": {"ms_per_step": attn_ms, "gbs": attn_bytes() / (attn_ms * 1e-3) / 1e9,
+                          "frac_hbm": attn_bytes() / (attn_ms * 1e-3) / 1e9 / peaks["hbm"]},
+            "quantize": {"ms_per_step": quant_ms, "gbs": quant_bytes / (quant_ms * 1e-3) / 1e9,
+                         "frac_hbm": quant_bytes / (quant_ms * 1e-3) / 1e9 / peaks["hbm"]},
+        },
+    }
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            out["cpu_baseline"] = cpu_baseline()
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------ oracle arm
+def oracle_step_sample(rows=2048, attn_rows=2048, hs=32):
+    """Times the oracle, as it stands, on a bounded sample of one step; returns (seconds scaled to a
+    full step, description)."""
+    from oracle import calibration as oc, linear as ol, attention as oa
+    t_full = 0.0
+    for key, C in INPUT_C.items():
+        Xcal = synth.activations(SEED, 100 + ord(key), 1, TOKENS, C)
+        gr = oc.calibrate(Xcal[:1024], 1024, 8, 8, dim_select=oc.DIM_CHANNEL)
+        X = synth.activations(SEED, 10 + ord(key), 1, rows, C)
+        t0 = time.perf_counter()
+        codes, s, z = ol.quantize_dynamic_token(X, gr.col_group, gr.G, 8)
+        t_q = time.perf_counter() - t0
+        t_l = 0.0
+        for i, (name, N, K, k2) in enumerate(LINEARS):
+            if k2 != key:
+                continue
+            wq, sw = ol.weight_rtn(synth.weights(SEED, 200 + i, N, K), 8)
+            bias = synth.bias(SEED, 300 + i, N)
+            t0 = time.perf_counter()
+            ol.group_linear(codes, s, z, gr.col_group, wq, sw, bias)
+            t_l += time.perf_counter() - t0
+        t_full += (t_q + t_l) * (M / rows)
+    a = ATT
+    Q, K, V = synth.attention_inputs(SEED, 1, a["H"], attn_rows, a["nk"], a["d"])
+    t0 = time.perf_counter()
+    oa.cross_attn_logq(Q, K, V, a["bits"])
+    t_full += (time.perf_counter() - t0) * (a["B"] * a["nq"] / attn_rows)
+    c = CONV
+
+    Xcal = synth.activations(SEED, 150, 1, hs * c["w"], c["c"], token_outliers=False)
+    gr = oc.calibrate(Xcal, hs * c["w"], 6, 16, dim_select=oc.DIM_CHANNEL)
+    X = synth.activations(SEED, 60, 1, hs * c["w"], c["c"], token_outliers=False)
+    wq, sw = ol.weight_rtn(synth.conv_weights(SEED, 250, c["N"], c["c"]), 4)
+    t0 = time.perf_counter()
+    codes, s, z = ol.quantize_static(X, gr, 0)
+    ol.group_conv3x3(codes.reshape(1, hs, c["w"], c["c"]), gr.scale[0][0], gr.zp[0][0], gr.col_group, wq, sw,
+                     synth.bias(SEED, 350, c["N"]))
+    t_full += (time.perf_counter() - t0) * (c["n"] * c["h"] / hs)
+    desc = (f"{rows} of {M} token rows of every linear (+ their quantizer), {attn_rows} of {a['B'] * a['nq']} "
+            f"query rows of the attention (all heads), {hs} of {c['n'] * c['h']} image rows of the conv; "
+            "time scaled to the full step by rows")
+    return t_full, desc
+
+
+def cpu_baseline():
+    t, desc = oracle_step_sample()
+    return {"value": gemm_ops() / t / 1e12, "unit": "TOPS", "cores": 1, "kind": "oracle", "sample": desc,
+            "est_seconds_per_step": t}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    for _ in range(max(0, min(args.warmup, 1))):
+        oracle_step_sample(rows=32, attn_rows=64)
+    ts, desc = [], ""
+    for _ in range(max(1, min(args.steps, 3))):
+        t, desc = oracle_step_sample()
+        ts.append(t)
+    t = float(np.mean(ts))
+    v = gemm_ops() / t / 1e12
+    print(json.dumps({
+        "impl": "reference", "metric": "group-quant GEMM TOPS & %INT8 peak; log-quant cross-attn GB/s & %HBM",
+        "value": v, "unit": "TOPS", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": len(ts),
+        "warmup": max(0, min(args.warmup, 1)), "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int64/f64", "data": "synthetic", "config": {"workload": WORKLOAD},
+        "cpu_baseline": {"value": v, "unit": "TOPS", "cores": 1, "kind": "oracle", "sample": desc},
+        "e2e": {"value": v, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -64,10 +64,16 @@ def cross_attn_logq(Q, K, V, bits, gran=PER_PROMPT, fixed_scale=None):
         s = np.maximum(np.asarray(fixed_scale, dtype=np.float64).reshape(-1, 1, 1, 1), FLT_MIN)
     s_full = np.broadcast_to(s, A.shape[:-1] + (1,))
     codes = log_quantize(A[..., 1:], s_full, bits)
+    return split_product(A, codes, s, V), codes, s, A
+
+
+def split_product(A, codes, s, V):
+    """Eq. 9: A_hat V = A[:, 0] V[0] + (s 2^-codes) V[1:], fp64, for given codes [B, H, nq, nk-1]."""
+    V = np.asarray(V, dtype=np.float64)
+    s_full = np.broadcast_to(s, A.shape[:-1] + (1,))
     A_hat_rest = log_dequantize(codes, s_full)
-    O = (np.einsum("bhq,bhd->bqhd", A[..., 0], V[:, 0])
-         + np.einsum("bhqk,bkhd->bqhd", A_hat_rest, V[:, 1:]))
-    return O, codes, s, A
+    return (np.einsum("bhq,bhd->bqhd", A[..., 0], V[:, 0])
+            + np.einsum("bhqk,bkhd->bqhd", A_hat_rest, V[:, 1:]))
 
 
 def attention_reference(Q, K, V):

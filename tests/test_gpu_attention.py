@@ -22,7 +22,13 @@ def _compare(torch, b, Q, K, V, bits, gran=0, fixed=None, code_frac=1e-4, out_re
     assert diff.max() <= 1, "a code differs by more than one level"
     frac = (diff != 0).mean()
     assert frac <= code_frac, f"{frac:.2e} of the codes differ"
-    check_output(O, O_ref, out_rel)
+    # A score that sits on a rounding boundary may take either neighbouring level (softmax rounding);
+    # one flipped level moves the output by up to half that score times |V|.  Rows whose codes all agree
+    # are held to the oracle's output; the others to Eq. 9 evaluated with the codes the kernel chose.
+    O_alt = oa.split_product(A, c, s_ref, V)
+    flipped = (diff != 0).any(axis=-1).transpose(0, 2, 1)          # [B, nq, H]
+    assert np.array_equal(O_alt[~flipped], O_ref[~flipped])
+    check_output(O, O_alt, out_rel)
     return frac
 
 
