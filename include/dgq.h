@@ -171,6 +171,37 @@ dgq_status dgq_cross_attn_logq(const void* Q, const void* K, const void* V, int 
                                size_t workspace_bytes, void* stream);
 dgq_status dgq_cross_attn_workspace_bytes(int B, int H, int nq, int nk, int d, size_t* bytes);
 
+/* ---------------------------------------------------------------- cross-attention without a caller workspace
+ * (The paper has no counterpart: this is a deployment convenience of this library.)
+ * Same computation, arguments and results as dgq_cross_attn_logq, for callers that
+ * have no way to obtain device memory for the workspace: code running inside a
+ * region where allocation is forbidden (a plugin or runtime callback that is only
+ * handed its input and output buffers, a real-time loop that must not call the
+ * allocator, a host that has already committed all device memory).  The scratch
+ * space lives in a fixed array inside the library image instead:
+ *   - DGQ_NOALLOC_SCRATCH_BYTES of device memory are held by every GPU that loads
+ *     the library, from load until the process exits, whether or not this call is
+ *     ever used;
+ *   - the problem must satisfy B * H * nq <= DGQ_NOALLOC_MAX_ROWS and
+ *     B * H <= DGQ_NOALLOC_MAX_HEADS, else DGQ_ERR_WORKSPACE is returned and
+ *     nothing is launched;
+ *   - the first call on each device looks up the device address of the array
+ *     (with that device current) and remembers it; make that first call before
+ *     starting any stream capture.  Later calls only enqueue work on `stream`;
+ *   - the call itself performs no allocation and frees nothing;
+ *   - all calls on a device share the one array.  It still holds the previous
+ *     call's statistics on entry; the part that must start clean is reset on
+ *     `stream` before the kernels run.  Two calls whose kernels can overlap on the
+ *     GPU (different streams without an ordering between them) race on it:
+ *     serialise them, or use dgq_cross_attn_logq with separate workspaces.
+ * Errors: those of dgq_cross_attn_logq. */
+#define DGQ_NOALLOC_MAX_ROWS (1 << 18)
+#define DGQ_NOALLOC_MAX_HEADS 256
+#define DGQ_NOALLOC_SCRATCH_BYTES (1024 + 8 * DGQ_NOALLOC_MAX_ROWS)
+dgq_status dgq_cross_attn_logq_noalloc(const void* Q, const void* K, const void* V, int B, int H, int nq, int nk,
+                                       int d, int score_bits, int scale_gran, const float* fixed_scale, void* O,
+                                       float* scale_out, uint8_t* codes_out, void* stream);
+
 /* ---------------------------------------------------------------- status
  * Synchronises the current device and returns the device status word of the
  * current device in *status (DGQ_OK, or the first error a kernel recorded),

@@ -27,7 +27,7 @@ EXPORTS = [
     "dgq_calibrate_groups", "dgq_groups_from_host", "dgq_groups_destroy", "dgq_groups_info",
     "dgq_groups_export", "dgq_quantize_act", "dgq_weight_prepare", "dgq_weight_from_codes",
     "dgq_weight_destroy", "dgq_weight_export", "dgq_linear", "dgq_cross_attn_logq",
-    "dgq_cross_attn_workspace_bytes", "dgq_device_status", "dgq_status_string", "dgq_launch_count",
+    "dgq_cross_attn_workspace_bytes", "dgq_cross_attn_logq_noalloc", "dgq_device_status", "dgq_status_string", "dgq_launch_count",
 ]
 
 
@@ -274,3 +274,27 @@ def cross_attn_logq(Q, K, V, score_bits=8, scale_gran=SCALE_PER_PROMPT, fixed_sc
                                    _ptr(scale), _ptr(codes), _ptr(ws), C.c_size_t(ws.numel()), _stream(stream))
     _check(st, "dgq_cross_attn_logq")
     return O, scale, codes
+
+
+NOALLOC_MAX_ROWS = 1 << 18
+NOALLOC_MAX_HEADS = 256
+
+
+def cross_attn_logq_noalloc(Q, K, V, O, score_bits=8, scale_gran=SCALE_PER_PROMPT, fixed_scale=None,
+                            scale_out=None, codes_out=None, stream=None):
+    """dgq_cross_attn_logq_noalloc: the same attention for callers that cannot provide a workspace.
+
+    Every buffer, the output included, comes from the caller; neither this wrapper nor the
+    library allocates.  The scratch is a fixed array inside the library, shared by all calls on a
+    device, so calls that may overlap on the GPU must be serialised.  Limits: B * H * nq <=
+    NOALLOC_MAX_ROWS and B * H <= NOALLOC_MAX_HEADS (status 4 beyond them).  The first call on a
+    device should come before any stream capture.
+    """
+    B, nq, H, d = Q.shape
+    nk = K.shape[1]
+    st = lib().dgq_cross_attn_logq_noalloc(_ptr(Q), _ptr(K), _ptr(V), C.c_int(B), C.c_int(H), C.c_int(nq),
+                                           C.c_int(nk), C.c_int(d), C.c_int(score_bits), C.c_int(scale_gran),
+                                           _ptr(fixed_scale), _ptr(O), _ptr(scale_out), _ptr(codes_out),
+                                           _stream(stream))
+    _check(st, "dgq_cross_attn_logq_noalloc")
+    return O

@@ -1,6 +1,7 @@
 // Single translation unit of the DGQ library (one device status word, no relocatable device code).
 #include <climits>
 #include <cmath>
+#include <mutex>
 
 #include "common.cuh"
 #include "groups.cuh"
@@ -8,6 +9,44 @@
 #include "weights.cuh"
 #include "linear.cuh"
 #include "attention.cuh"
+
+// ---------------------------------------------------------------------------------------------
+// Cross-attention for callers that cannot allocate a workspace: the scratch is this fixed array
+// in the library image (one copy per GPU that loads the library).  In host code the name
+// `g_noalloc_scratch` is only a handle for the runtime, never a device address; the address that
+// kernels may use comes from cudaGetSymbolAddress, looked up once per device.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[DGQ_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+std::mutex g_noalloc_mutex;
+void* g_noalloc_ptr[64] = {nullptr};  // device address of the scratch array, per device ordinal
+}  // namespace
+
+extern "C" dgq_status dgq_cross_attn_logq_noalloc(const void* Q, const void* K, const void* V, int B, int H, int nq,
+                                                  int nk, int d, int score_bits, int scale_gran,
+                                                  const float* fixed_scale, void* O, float* scale_out,
+                                                  uint8_t* codes_out, void* stream) {
+  if (B <= 0 || H <= 0 || nq <= 0) return DGQ_ERR_INVALID_ARG;
+  if ((int64_t)B * H > DGQ_NOALLOC_MAX_HEADS || (int64_t)B * H * nq > DGQ_NOALLOC_MAX_ROWS)
+    return DGQ_ERR_WORKSPACE;  // larger than the built-in scratch: use dgq_cross_attn_logq
+  int dev = 0;
+  DGQ_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return DGQ_ERR_UNSUPPORTED;
+  void* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {  // first call on this device, which is the current one
+      void* p = nullptr;
+      if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return DGQ_ERR_CUDA;
+      g_noalloc_ptr[dev] = p;
+    }
+    scratch = g_noalloc_ptr[dev];
+  }
+  // The workspace path resets the per-scope maxima on `stream` itself and overwrites every row
+  // statistic it later reads, so stale contents from an earlier call are harmless.
+  return dgq_cross_attn_logq(Q, K, V, B, H, nq, nk, d, score_bits, scale_gran, fixed_scale, O, scale_out,
+                             codes_out, scratch, (size_t)DGQ_NOALLOC_SCRATCH_BYTES, stream);
+}
 
 extern "C" dgq_status dgq_device_status(int* status) {
   if (!status) return DGQ_ERR_INVALID_ARG;
