@@ -393,6 +393,130 @@ def run_reference(args):
     }))
 
 
+# ------------------------------------------------------------------------------------------ single-kernel cases
+MICRO_CASES = {
+    # name: (kind, params)
+    "quant_8192x320": ("quant", dict(M=8192, P=4096, C=320, G=8, dynamic=1)),
+    "quant_8192x1280": ("quant", dict(M=8192, P=4096, C=1280, G=8, dynamic=1)),
+    "quant_32768x320": ("quant", dict(M=32768, P=4096, C=320, G=8, dynamic=1)),
+    "quant_32768x1280": ("quant", dict(M=32768, P=4096, C=1280, G=8, dynamic=1)),
+    "quant_static_32768x320": ("quant", dict(M=32768, P=4096, C=320, G=16, dynamic=0)),
+    "gemm_8192x320x320_w8": ("gemm", dict(M=8192, P=4096, N=320, C=320, G=8, wbits=8)),
+    "gemm_8192x2560x320_w8": ("gemm", dict(M=8192, P=4096, N=2560, C=320, G=8, wbits=8)),
+    "gemm_8192x320x1280_w8": ("gemm", dict(M=8192, P=4096, N=320, C=1280, G=8, wbits=8)),
+    "gemm_32768x320x1280_w4": ("gemm", dict(M=32768, P=4096, N=320, C=1280, G=8, wbits=4)),
+    "gemm_8192x640x640_w4": ("gemm", dict(M=8192, P=1024, N=640, C=640, G=8, wbits=4)),
+    "gemm_8192x5120x640_w4": ("gemm", dict(M=8192, P=1024, N=5120, C=640, G=8, wbits=4)),
+    "gemm_8192x640x2560_w4": ("gemm", dict(M=8192, P=1024, N=640, C=2560, G=8, wbits=4)),
+    "gemm_2048x1280x5120_w4": ("gemm", dict(M=2048, P=256, N=1280, C=5120, G=8, wbits=4)),
+    "conv_2x64x64x320": ("conv", dict(n=2, h=64, w=64, C=320, N=320, G=16)),
+    "conv_8x64x64x320": ("conv", dict(n=8, h=64, w=64, C=320, N=320, G=16)),
+    "conv_8x32x32x640": ("conv", dict(n=8, h=32, w=32, C=640, N=640, G=16)),
+    "conv_8x16x16x1280": ("conv", dict(n=8, h=16, w=16, C=1280, N=1280, G=16)),
+    "attn_2x4096x40": ("attn", dict(B=2, H=8, nq=4096, nk=77, d=40)),
+    "attn_8x4096x40": ("attn", dict(B=8, H=8, nq=4096, nk=77, d=40)),
+    "attn_8x1024x80": ("attn", dict(B=8, H=8, nq=1024, nk=77, d=80)),
+    "attn_8x256x160": ("attn", dict(B=8, H=8, nq=256, nk=77, d=160)),
+}
+
+
+def run_micro(args):
+    """Times single kernels: each case is captured as a CUDA graph of back-to-back launches that
+    rotate over buffer sets larger than L2, replayed and timed with CUDA events."""
+    import torch
+    from paper_2501_04304_b200 import binding as b
+    torch.cuda.set_device(0)
+    peaks = measured_peaks()
+    names = [n for n in MICRO_CASES if args.micro == "all" or n.startswith(args.micro)]
+    for name in names:
+        kind, p = MICRO_CASES[name]
+        fns, algo_bytes, algo_ops = [], 0.0, 0.0
+        if kind in ("quant", "gemm", "conv"):
+            conv = None
+            if kind == "conv":
+                P, M, C, bits, tok = p["h"] * p["w"], p["n"] * p["h"] * p["w"], p["C"], 6, False
+                conv = (p["n"], p["h"], p["w"], C)
+            else:
+                P, M, C, bits, tok = p["P"], p["M"], p["C"], 8, True
+            Xcal = torch.from_numpy(synth.activations(SEED, 100, 2, P, C, token_outliers=tok)).cuda()
+            g = b.calibrate_groups(Xcal, P, bits, p["G"], b.DIM_CHANNEL)
+            Xh = synth.activations(SEED, 1, M // P, P, C, token_outliers=tok)
+            per_set = M * C * 2 + M * g.K_pad + (M * p.get("N", 0) * 2)
+            n_sets = max(2, int(3 * 126e6 // per_set) + 1)
+            dyn = kind == "gemm" or (kind == "quant" and p["dynamic"])
+            mode = b.MODE_DYNAMIC_TOKEN if dyn else b.MODE_STATIC
+            layout = b.CODES_S8_CENTRED if kind == "conv" else b.CODES_U8
+            sets = []
+            for _ in range(n_sets):
+                X = torch.from_numpy(Xh).cuda()
+                Xq = torch.empty((M, g.K_pad), dtype=torch.uint8, device="cuda")
+                ds = torch.empty((M, g.G), dtype=torch.float32, device="cuda") if dyn else None
+                dz = torch.empty((M, g.G), dtype=torch.int32, device="cuda") if dyn else None
+                b.quantize_act_into(g, X, Xq, ds, dz, mode=mode, layout=layout)
+                Y = torch.empty((M, p["N"]), dtype=torch.float16, device="cuda") if kind != "quant" else None
+                sets.append((X, Xq, ds, dz, Y))
+            if kind == "quant":
+                fns = [lambda s=s: b.quantize_act_into(g, s[0], s[1], s[2], s[3], mode=mode, layout=layout) for s in sets]
+                algo_bytes = 3.0 * M * C + (8.0 * M * g.G if dyn else 0)
+            else:
+                if kind == "conv":
+                    W = torch.from_numpy(synth.conv_weights(SEED, 2, p["N"], C)).cuda()
+                    w = b.weight_prepare(g, W, 4, conv=conv)
+                    kreal, wb = 9 * C, 4
+                else:
+                    W = torch.from_numpy(synth.weights(SEED, 2, p["N"], C)).cuda()
+                    w = b.weight_prepare(g, W, p["wbits"])
+                    kreal, wb = C, p["wbits"]
+                bias = torch.from_numpy(synth.bias(SEED, 3, p["N"])).cuda()
+                fns = [lambda s=s: b.linear(g, w, s[1], mode=mode, layout=layout, dyn_scale=s[2], dyn_zp=s[3],
+                                            bias=bias, out=s[4], conv=conv) for s in sets]
+                algo_ops = 2.0 * M * p["N"] * kreal
+                algo_bytes = M * C + p["N"] * kreal * wb / 8 + 2.0 * M * p["N"]
+            extra = {"K_pad": g.K_pad, "G": g.G}
+        else:
+            a = p
+            Q, K, V = synth.attention_inputs(SEED, a["B"], a["H"], a["nq"], a["nk"], a["d"])
+            per_set = 2 * Q.size * 2
+            n_sets = max(2, int(3 * 126e6 // per_set) + 1)
+            ws_bytes = b.cross_attn_workspace_bytes(a["B"], a["H"], a["nq"], a["nk"], a["d"])
+            sets = [(torch.from_numpy(Q).cuda(), torch.from_numpy(K).cuda(), torch.from_numpy(V).cuda(),
+                     torch.empty(Q.shape, dtype=torch.float16, device="cuda"),
+                     torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")) for _ in range(n_sets)]
+            fns = [lambda s=s: b.cross_attn_logq(s[0], s[1], s[2], 8, out=s[3], workspace=s[4]) for s in sets]
+            algo_bytes = 2.0 * Q.size * 2 + 2.0 * K.size * 2
+            extra = {}
+        reps = max(1, 24 // len(fns))
+        for f in fns:
+            f()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        stream = torch.cuda.Stream()
+        with torch.cuda.stream(stream):
+            with torch.cuda.graph(graph, stream=stream):
+                for _ in range(reps):
+                    for f in fns:
+                        f()
+        n_launch = reps * len(fns)
+        torch.cuda.synchronize()
+        times = []
+        for _ in range(3 + args.steps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            graph.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1) * 1e3 / n_launch)
+        us = float(np.median(times[3:]))
+        rec = {"case": name, "us": us, "gbs": algo_bytes / us / 1e3, "frac_hbm": algo_bytes / us / 1e3 / peaks["hbm"],
+               "sets": len(fns), **extra}
+        if algo_ops:
+            rec["tops"] = algo_ops / us / 1e6
+            rec["frac_int8_peak"] = rec["tops"] / (2 * peaks["bf16"])
+        assert b.device_status() == 0
+        print(json.dumps(rec), flush=True)
+        del sets, fns, graph
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -400,8 +524,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--micro", default=None, help="time single kernels: 'all' or a case-name prefix")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.micro:
+        run_micro(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_cuda(args)

@@ -223,6 +223,8 @@ static std::vector<int> group_vectors(const std::vector<double>& vmin, const std
 }
 
 // ------------------------------------------------------------------ host: object plumbing
+constexpr int GROUP_MIN_PAD = 8;
+
 static void groups_free_device(dgq_groups* g) {
   cudaFree(g->d_perm);
   cudaFree(g->d_chunk_group);
@@ -234,7 +236,9 @@ static void groups_free_device(dgq_groups* g) {
 }
 
 // Padded, group-contiguous code layout: members of each group in ascending channel order, every
-// group padded to a multiple of DGQ_K_ATOM positions.
+// group padded to a multiple of DGQ_K_ATOM positions with at least GROUP_MIN_PAD padding positions.
+// The padding carries the cell's zero-point as its code; the weight side stores -wsum spread over
+// those positions, so the integer product already contains the zero-point term of Eq. 1.
 static dgq_status groups_build_layout(dgq_groups* g) {
   g->group_off.assign(g->G + 1, 0);
   g->perm.clear();
@@ -242,6 +246,7 @@ static dgq_status groups_build_layout(dgq_groups* g) {
     g->group_off[k] = (int32_t)g->perm.size();
     for (int c = 0; c < g->C; ++c)
       if (g->col_group[c] == k) g->perm.push_back(c);
+    for (int i = 0; i < GROUP_MIN_PAD; ++i) g->perm.push_back(-1);
     while (g->perm.size() % DGQ_K_ATOM) g->perm.push_back(-1);
   }
   g->K_pad = (int)g->perm.size();

@@ -5,13 +5,23 @@
 // (Eq. 1's de-quantizer with the group parameters of Eq. 6) fused in.
 //
 // CTA = one 128-row output tile x BN columns, persistent over tiles.  Warp roles:
-//   warps 0-7   epilogue: lane quarter = warp & 3 (the TMEM lanes a warp may read), column half = warp >> 2
-//   warp  8     TMA producer (one elected lane): A code tile and B weight tile per 128-byte K stage
-//   warp  9     MMA issuer (one elected lane) and TMEM allocator
-//   warps 10-13 (4-bit weights only) unpack packed nibbles from global memory into the B stage
+//   warps 0-15  epilogue: lane quarter = warp & 3 (the TMEM lanes a warp may read), column slice = warp >> 2
+//   warp  16    TMA producer (one elected lane): A code tile and B weight tile per 128-byte K stage
+//   warp  17    MMA issuer (one elected lane) and TMEM allocator
+//   warps 18-21 (4-bit weights only) unpack packed nibbles from global memory into the B stage
 // K runs over 32-code atoms; a stage holds four atoms.  Group segments are multiples of one atom,
 // so the issuer moves to the next TMEM accumulator between two atoms, commits the finished one to
 // the epilogue and keeps going while the epilogue drains it.
+//
+// Zero-points: the padding positions of a group carry the code Z on the activation side and
+// -wsum_g[o] (spread over the positions) on the weight side, so acc_g already equals
+// acc_g - Z wsum_g and the epilogue is one convert and one FMA per element and group.  The
+// epilogue only adds a correction for the rare rows whose Z falls outside the code range (the
+// stored padding code is then the clamped Z) and for groups whose padding could not hold all of
+// wsum (flagged in `res_mask`).
+//
+// Output: the fp16 tile is staged in shared memory in 64-byte-swizzled panels of 32 columns and
+// written with TMA stores, which also clip the ragged last row and column tiles.
 // Linear layers: A and B stages are 128-byte-swizzled tiles fetched with one TMA box each.
 // 3x3 conv (implicit GEMM): the reduction order is group-major, then filter tap, then channel
 // atom; every A atom is its own 32-byte-swizzled 4-D TMA box of the NHWC code tensor shifted by
@@ -23,7 +33,12 @@
 namespace dgq {
 
 constexpr int GEMM_BM = 128;
-constexpr int GEMM_EPI_WARPS = 8;
+constexpr int GEMM_EPI_WARPS = 16;
+constexpr int GEMM_EPI_THREADS = GEMM_EPI_WARPS * 32;
+constexpr int GEMM_WARP_TMA = 16;
+constexpr int GEMM_WARP_MMA = 17;
+constexpr int GEMM_THREADS_W8 = 18 * 32;
+constexpr int GEMM_THREADS_W4 = 22 * 32;
 constexpr int GEMM_A_STAGE = GEMM_BM * 128;  // bytes
 constexpr int GEMM_SMEM_LIMIT = 227 * 1024;
 
@@ -31,12 +46,14 @@ template <int BN>
 struct GemmCfg {
   static constexpr int B_STAGE = BN * 128;
   static constexpr int STAGE = GEMM_A_STAGE + B_STAGE;
-  static constexpr int STAGES_RAW = (GEMM_SMEM_LIMIT - 3072) / STAGE;
+  static constexpr int OUT_BYTES = GEMM_BM * BN * 2;  // fp16 staging of one output tile
+  static constexpr int MISC_BYTES = 2048 + BN * 8;    // barriers + sw / bias of the tile's columns
+  static constexpr int STAGES_RAW = (GEMM_SMEM_LIMIT - 1024 - OUT_BYTES - MISC_BYTES) / STAGE;
   static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
   static constexpr int NACC_RAW = 512 / BN;
   static constexpr int NACC = NACC_RAW > 4 ? 4 : NACC_RAW;
-  static constexpr int CH = BN / 2;  // columns per epilogue thread
-  static constexpr int SMEM = STAGES * STAGE + 2048 + 1024;
+  static constexpr int CW = BN / 4;  // columns per epilogue thread
+  static constexpr int SMEM = STAGES * STAGE + OUT_BYTES + MISC_BYTES + 1024;
   static_assert(BN % 32 == 0 && BN <= 256, "BN must be a multiple of 32 up to 256");
   static_assert(NACC >= 2, "need two accumulators to overlap the epilogue");
   static_assert(NACC * BN <= 512, "tensor memory has 512 columns");
@@ -49,19 +66,20 @@ struct GemmArgs {
   int n_tiles_m, n_tiles_n;
   uint32_t idesc;
   int use_zp;                 // 0 for zero-centred codes
+  int code_max;               // 2^b - 1
+  uint32_t res_mask;          // groups whose padding did not absorb all of wsum
   int per_token;              // 1: scale rows indexed by token, 0: by row_group[token mod P]
   const float* scale;         // [rows][G]
   const int32_t* zp;          // [rows][G]
   const int32_t* row_group;   // [P]
   const float* sw;            // [N_pad]
   const float* wsum;          // [G][N_pad]
+  const float* wres;          // [G][N_pad]
   const __half* bias;         // [N] or null
-  __half* Y;
-  int64_t ldy;
   const uint8_t* w_packed;    // 4-bit weights [N_pad][Kt/2]
   int seg_end[DGQ_MAX_GROUPS];    // end atom of every group segment
   // conv
-  int conv_W, conv_H, box_w, box_h, box_n;
+  int conv_W, conv_H;
   int grp_atoms[DGQ_MAX_GROUPS];  // channel atoms of every group
   int grp_chan0[DGQ_MAX_GROUPS];  // first padded channel position of every group
 };
@@ -71,14 +89,24 @@ struct __align__(8) GemmShared {
   uint64_t empty[8];
   uint64_t acc_full[4];
   uint64_t acc_empty[4];
+  uint64_t epi_bar;
   uint32_t tmem_base;
   int abort_flag;
 };
 
+// Barrier among the epilogue warps with a bounded wait (one arrival per warp).
+__device__ __forceinline__ bool epi_sync(uint64_t* bar, uint32_t& phase, int lane, volatile int* abort_flag) {
+  __syncwarp();
+  if (lane == 0) mbar_arrive(bar);
+  const bool ok = __all_sync(0xffffffffu, mbar_wait(bar, phase & 1u, abort_flag));
+  phase ^= 1u;
+  return ok;
+}
+
 template <int BN, bool W4, bool CONV>
-__global__ void __launch_bounds__(W4 ? 448 : 320, 1)
+__global__ void __launch_bounds__(W4 ? GEMM_THREADS_W4 : GEMM_THREADS_W8, 1)
 gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const __grid_constant__ GemmArgs a) {
+               const __grid_constant__ CUtensorMap tmY, const __grid_constant__ GemmArgs a) {
   using Cfg = GemmCfg<BN>;
   constexpr int STAGES = Cfg::STAGES;
   constexpr int NACC = Cfg::NACC;
@@ -87,7 +115,10 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                                          ~uintptr_t(1023));
   unsigned char* smA = smem;
   unsigned char* smB = smem + STAGES * GEMM_A_STAGE;
-  GemmShared* sh = reinterpret_cast<GemmShared*>(smem + STAGES * Cfg::STAGE);
+  unsigned char* smOut = smem + STAGES * Cfg::STAGE;  // 1024-byte aligned: every stage size is
+  GemmShared* sh = reinterpret_cast<GemmShared*>(smOut + Cfg::OUT_BYTES);
+  float* sw_s = reinterpret_cast<float*>(smOut + Cfg::OUT_BYTES + 2048);
+  float* bias_s = sw_s + BN;
   volatile int* abort_flag = &sh->abort_flag;
 
   const int warp = threadIdx.x >> 5;
@@ -105,10 +136,11 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       mbar_init(&sh->acc_full[i], 1);
       mbar_init(&sh->acc_empty[i], GEMM_EPI_WARPS);
     }
+    mbar_init(&sh->epi_bar, GEMM_EPI_WARPS);
     sh->abort_flag = 0;
     fence_barrier_init();
   }
-  if (warp == 9) {
+  if (warp == GEMM_WARP_MMA) {
     tmem_alloc(&sh->tmem_base, 512);
     tmem_relinquish();
   }
@@ -117,11 +149,12 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   tc_fence_after();
   const uint32_t tmem_base = sh->tmem_base;
 
-  if (warp == 8) {
+  if (warp == GEMM_WARP_TMA) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&tmA);
       if (!W4) tma_prefetch_desc(&tmB);
+      tma_prefetch_desc(&tmY);
       uint32_t it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
@@ -166,7 +199,7 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
       }
     }
-  } else if (warp == 9) {
+  } else if (warp == GEMM_WARP_MMA) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       uint32_t it = 0, acc_it = 0;
@@ -213,108 +246,143 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   } else if (warp < GEMM_EPI_WARPS) {
     // ------------------------------------------------------------ epilogue
-    constexpr int CH = Cfg::CH;
-    const int q = warp & 3, half = warp >> 2;
-    uint32_t acc_it = 0;
+    constexpr int CW = Cfg::CW;
+    constexpr int NCH = CW / 8;
+    const int q = warp & 3, sl = warp >> 2;
+    const int r_tile = q * 32 + lane;  // row inside the tile = TMEM lane
+    uint32_t acc_it = 0, sync_phase = 0;
     bool ok = true;
+    bool stored = false;
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
       const int tm = tile / a.n_tiles_n, tn = tile - tm * a.n_tiles_n;
-      const int64_t row = (int64_t)tm * GEMM_BM + q * 32 + lane;
+      const int n0 = tn * BN;
+      const int64_t row = (int64_t)tm * GEMM_BM + r_tile;
       const int64_t row_c = row < a.M ? row : a.M - 1;
-      const int col0 = tn * BN + half * CH;
+      const int col0 = n0 + sl * CW;
       const int64_t prow = a.per_token ? row_c : (int64_t)a.row_group[row_c % a.P];
       const float* srow = a.scale + prow * a.G;
       const int32_t* zrow = a.zp + prow * a.G;
-      float y[CH];
+      // per-column constants of this tile (read again only after the next barrier)
+      for (int i = threadIdx.x; i < BN; i += GEMM_EPI_THREADS) {
+        const int col = n0 + i;
+        sw_s[i] = col < a.N_pad ? __ldg(a.sw + col) : 0.f;
+        bias_s[i] = (a.bias != nullptr && col < a.N) ? __half2float(a.bias[col]) : 0.f;
+      }
+      float y[CW];
 #pragma unroll
-      for (int i = 0; i < CH; ++i) y[i] = 0.f;
+      for (int i = 0; i < CW; ++i) y[i] = 0.f;
+      float s_next = __ldg(srow);
       for (int g = 0; g < a.G && ok; ++g, ++acc_it) {
-        const float s = __ldg(srow + g);
-        const float c = a.use_zp ? -s * (float)__ldg(zrow + g) : 0.f;
+        const float s = s_next;
+        if (g + 1 < a.G) s_next = __ldg(srow + g + 1);
+        float c1 = 0.f, c2 = 0.f;
+        if (a.use_zp) {
+          const int Z = __ldg(zrow + g);
+          const int Zc = min(max(Z, 0), a.code_max);
+          c1 = -s * (float)(Z - Zc);
+          c2 = ((a.res_mask >> g) & 1u) ? -s * (float)Zc : 0.f;
+        }
         const int ab = acc_it % NACC;
         ok = __all_sync(0xffffffffu, mbar_wait(&sh->acc_full[ab], (acc_it / NACC) & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
-        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * BN + half * CH);
-        const float* ws = a.wsum + (size_t)g * a.N_pad + col0;
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * BN + sl * CW);
+        // Two register buffers: the load of chunk k + 1 is in flight while chunk k is converted and
+        // accumulated.  The accumulator is handed back as soon as its last chunk is in registers.
+        uint32_t rb[2][8];
+        tmem_ld8(taddr, rb[0]);
 #pragma unroll
-        for (int cc = 0; cc < CH; cc += 16) {
-          uint32_t r[16];
-          tmem_ld16(taddr + cc, r);
+        for (int k = 0; k < NCH; ++k) {
           tmem_ld_wait();
+          if (k + 1 < NCH) {
+            tmem_ld8(taddr + (k + 1) * 8, rb[(k + 1) & 1]);
+          } else {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh->acc_empty[ab]);
+          }
 #pragma unroll
-          for (int i = 0; i < 16; ++i) y[cc + i] = fmaf(s, (float)(int)r[i], y[cc + i]);
-          if (a.use_zp) {
+          for (int i = 0; i < 8; ++i) y[k * 8 + i] = fmaf(s, (float)(int)rb[k & 1][i], y[k * 8 + i]);
+        }
+        if (__any_sync(0xffffffffu, c1 != 0.f || c2 != 0.f)) {
+          const float4* ws = reinterpret_cast<const float4*>(a.wsum + (size_t)g * a.N_pad + col0);
+          const float4* wr = reinterpret_cast<const float4*>(a.wres + (size_t)g * a.N_pad + col0);
 #pragma unroll
-            for (int i = 0; i < 16; i += 4) {
-              const float4 w4 = __ldg(reinterpret_cast<const float4*>(ws + cc + i));
-              y[cc + i] = fmaf(c, w4.x, y[cc + i]);
-              y[cc + i + 1] = fmaf(c, w4.y, y[cc + i + 1]);
-              y[cc + i + 2] = fmaf(c, w4.z, y[cc + i + 2]);
-              y[cc + i + 3] = fmaf(c, w4.w, y[cc + i + 3]);
-            }
+          for (int i = 0; i < CW; i += 4) {
+            const float4 u = __ldg(ws + (i >> 2)), v = __ldg(wr + (i >> 2));
+            y[i] = fmaf(c1, u.x, fmaf(c2, v.x, y[i]));
+            y[i + 1] = fmaf(c1, u.y, fmaf(c2, v.y, y[i + 1]));
+            y[i + 2] = fmaf(c1, u.z, fmaf(c2, v.z, y[i + 2]));
+            y[i + 3] = fmaf(c1, u.w, fmaf(c2, v.w, y[i + 3]));
           }
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sh->acc_empty[ab]);
       }
       if (!ok) break;
-      if (row < a.M) {
-        __half* yrow = a.Y + row * a.ldy;
+      // the previous tile's TMA stores must have finished reading the staging buffer
+      if (stored && threadIdx.x == 0) bulk_wait_read0();
+      ok = epi_sync(&sh->epi_bar, sync_phase, lane, abort_flag);
+      if (!ok) break;
 #pragma unroll
-        for (int i = 0; i < CH; i += 8) {
-          const int col = col0 + i;
-          if (col < a.N) {
-            const float4 s0 = __ldg(reinterpret_cast<const float4*>(a.sw + col));
-            const float4 s1 = __ldg(reinterpret_cast<const float4*>(a.sw + col + 4));
-            float b[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-            if (a.bias) {
-              const uint4 bv = __ldg(reinterpret_cast<const uint4*>(a.bias + col));
-              const __half2* bh = reinterpret_cast<const __half2*>(&bv);
+      for (int j = 0; j < NCH; ++j) {
+        const int cl = sl * CW + j * 8;  // first tile column of this 16-byte chunk
+        uint4 o;
+        __half2* oh = reinterpret_cast<__half2*>(&o);
 #pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                const float2 f = __half22float2(bh[k]);
-                b[2 * k] = f.x;
-                b[2 * k + 1] = f.y;
-              }
-            }
-            const float sw8[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-            uint4 o;
-            __half2* oh = reinterpret_cast<__half2*>(&o);
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              oh[k] = __floats2half2_rn(fmaf(sw8[2 * k], y[i + 2 * k], b[2 * k]),
-                                        fmaf(sw8[2 * k + 1], y[i + 2 * k + 1], b[2 * k + 1]));
-            *reinterpret_cast<uint4*>(yrow + col) = o;
-          }
-        }
+        for (int k = 0; k < 4; ++k)
+          oh[k] = __floats2half2_rn(fmaf(sw_s[cl + 2 * k], y[j * 8 + 2 * k], bias_s[cl + 2 * k]),
+                                    fmaf(sw_s[cl + 2 * k + 1], y[j * 8 + 2 * k + 1], bias_s[cl + 2 * k + 1]));
+        // panel of 32 columns = 64-byte rows, 16-byte chunk index XOR bits 1-2 of the row (64 B swizzle)
+        const int panel = cl >> 5, ch = (cl >> 3) & 3;
+        *reinterpret_cast<uint4*>(smOut + panel * (GEMM_BM * 64) + r_tile * 64 + ((ch ^ ((r_tile >> 1) & 3)) << 4)) = o;
       }
+      fence_proxy_async_smem();
+      ok = epi_sync(&sh->epi_bar, sync_phase, lane, abort_flag);
+      if (!ok) break;
+      if (threadIdx.x == 0) {
+#pragma unroll
+        for (int pnl = 0; pnl < BN / 32; ++pnl)
+          if (n0 + pnl * 32 < a.N) tma_store_2d(&tmY, smOut + pnl * (GEMM_BM * 64), n0 + pnl * 32, tm * GEMM_BM);
+        bulk_commit();
+      }
+      stored = true;
     }
+    if (stored && threadIdx.x == 0) bulk_wait0();
   } else if (W4) {
     // ------------------------------------------------------------ 4-bit weight unpack into the B stage
-    const int ut = threadIdx.x - 320;  // 0..127
+    constexpr int ITEMS = BN * 4 / 128;  // 16-byte packed pieces per thread and stage
+    const int ut = threadIdx.x - GEMM_THREADS_W8;  // 0..127
     uint32_t it = 0;
     bool ok = true;
     const int row_bytes = a.Kt >> 1;
+    uint4 pk[ITEMS];
+    auto fetch = [&](int tile, int ks) {
+      const int n0 = (tile % a.n_tiles_n) * BN;
+#pragma unroll
+      for (int e = 0; e < ITEMS; ++e) {
+        const int item = ut + e * 128;
+        const int r = item >> 2, qd = item & 3;  // B row, 16-byte packed quarter of the 64-byte row slice
+        const int kb = ks * 64 + qd * 16;
+        pk[e] = make_uint4(0u, 0u, 0u, 0u);
+        if (kb < row_bytes)
+          pk[e] = __ldg(reinterpret_cast<const uint4*>(a.w_packed + (size_t)(n0 + r) * row_bytes + kb));
+      }
+    };
+    if ((int)blockIdx.x < n_tiles) fetch(blockIdx.x, 0);
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-      const int tn = tile % a.n_tiles_n;
-      const int n0 = tn * BN;
       for (int ks = 0; ks < n_kstages && ok; ++ks, ++it) {
         const int s = it % STAGES;
         ok = __all_sync(0xffffffffu, mbar_wait(&sh->empty[s], ((it / STAGES) & 1) ^ 1, abort_flag));
         if (!ok) break;
         unsigned char* bst = smB + s * Cfg::B_STAGE;
-        for (int item = ut; item < BN * 4; item += 128) {
-          const int r = item >> 2, qd = item & 3;  // B row, 16-byte packed quarter of the 64-byte row slice
-          const int kb = ks * 64 + qd * 16;
-          uint4 pk = make_uint4(0u, 0u, 0u, 0u);
-          if (kb < row_bytes)
-            pk = __ldg(reinterpret_cast<const uint4*>(a.w_packed + (size_t)(n0 + r) * row_bytes + kb));
-          const uint4 c0 = make_uint4((pk.x << 4) & 0xF0F0F0F0u, pk.x & 0xF0F0F0F0u, (pk.y << 4) & 0xF0F0F0F0u,
-                                      pk.y & 0xF0F0F0F0u);
-          const uint4 c1 = make_uint4((pk.z << 4) & 0xF0F0F0F0u, pk.z & 0xF0F0F0F0u, (pk.w << 4) & 0xF0F0F0F0u,
-                                      pk.w & 0xF0F0F0F0u);
+#pragma unroll
+        for (int e = 0; e < ITEMS; ++e) {
+          const int item = ut + e * 128;
+          const int r = item >> 2, qd = item & 3;
+          const uint4 p4 = pk[e];
+          const uint4 c0 = make_uint4((p4.x << 4) & 0xF0F0F0F0u, p4.x & 0xF0F0F0F0u, (p4.y << 4) & 0xF0F0F0F0u,
+                                      p4.y & 0xF0F0F0F0u);
+          const uint4 c1 = make_uint4((p4.z << 4) & 0xF0F0F0F0u, p4.z & 0xF0F0F0F0u, (p4.w << 4) & 0xF0F0F0F0u,
+                                      p4.w & 0xF0F0F0F0u);
           // 128-byte swizzle: 16-byte chunk index XOR (row mod 8) inside every 8-row, 1024-byte group
           unsigned char* rowp = bst + (r >> 3) * 1024 + (r & 7) * 128;
           *reinterpret_cast<uint4*>(rowp + (((2 * qd) ^ (r & 7)) << 4)) = c0;
@@ -323,6 +391,9 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh->full[s]);
+        // the next stage's nibbles travel while the tensor core works on this one
+        if (ks + 1 < n_kstages) fetch(tile, ks + 1);
+        else if (tile + (int)gridDim.x < n_tiles) fetch(tile + gridDim.x, 0);
       }
     }
   }
@@ -337,7 +408,8 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     __syncthreads();
   }
-  if (warp == 9) {
+  if (warp == GEMM_WARP_MMA) {
+    __syncwarp();
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
   }
@@ -361,7 +433,8 @@ static EncodeTiledFn get_encode_fn() {
 }
 
 static bool encode_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides,
-                       const uint32_t* box, CUtensorMapSwizzle sw) {
+                       const uint32_t* box, CUtensorMapSwizzle sw,
+                       CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_UINT8) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
   cuuint64_t d[5];
@@ -373,14 +446,14 @@ static bool encode_map(CUtensorMap* m, const void* base, int rank, const uint64_
     es[i] = 1;
   }
   for (int i = 0; i + 1 < rank; ++i) st[i] = strides[i];
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void*>(base), d, st, b, es,
+  return fn(m, dtype, (cuuint32_t)rank, const_cast<void*>(base), d, st, b, es,
             CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 template <int BN, bool W4, bool CONV>
-static dgq_status launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& a, int grid,
-                              cudaStream_t stream) {
+static dgq_status launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
+                              const GemmArgs& a, int grid, cudaStream_t stream) {
   using Cfg = GemmCfg<BN>;
   static bool attr_set[64] = {false};
   int dev = 0;
@@ -390,7 +463,7 @@ static dgq_status launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, co
                                      Cfg::SMEM));
     if (dev < 64) attr_set[dev] = true;
   }
-  gq_gemm_kernel<BN, W4, CONV><<<grid, W4 ? 448 : 320, Cfg::SMEM, stream>>>(tmA, tmB, a);
+  gq_gemm_kernel<BN, W4, CONV><<<grid, W4 ? GEMM_THREADS_W4 : GEMM_THREADS_W8, Cfg::SMEM, stream>>>(tmA, tmB, tmY, a);
   g_launches += 1;
   DGQ_CUDA_OK(cudaGetLastError());
   return DGQ_OK;
@@ -398,12 +471,12 @@ static dgq_status launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, co
 
 template <int BN>
 static dgq_status launch_gemm_bn(bool w4, bool conv, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                                 const GemmArgs& a, int grid, cudaStream_t stream) {
+                                 const CUtensorMap& tmY, const GemmArgs& a, int grid, cudaStream_t stream) {
   if (w4)
-    return conv ? launch_gemm<BN, true, true>(tmA, tmB, a, grid, stream)
-                : launch_gemm<BN, true, false>(tmA, tmB, a, grid, stream);
-  return conv ? launch_gemm<BN, false, true>(tmA, tmB, a, grid, stream)
-              : launch_gemm<BN, false, false>(tmA, tmB, a, grid, stream);
+    return conv ? launch_gemm<BN, true, true>(tmA, tmB, tmY, a, grid, stream)
+                : launch_gemm<BN, true, false>(tmA, tmB, tmY, a, grid, stream);
+  return conv ? launch_gemm<BN, false, true>(tmA, tmB, tmY, a, grid, stream)
+              : launch_gemm<BN, false, false>(tmA, tmB, tmY, a, grid, stream);
 }
 
 }  // namespace dgq
@@ -442,12 +515,13 @@ extern "C" dgq_status dgq_linear(const dgq_groups* g, const dgq_weight* w, int t
   a.G = g->G;
   a.P = g->P;
   a.use_zp = (layout == DGQ_CODES_U8);
+  a.code_max = (1 << g->bits) - 1;
+  a.res_mask = w->res_mask;
+  a.wres = w->d_wres;
   a.row_group = g->d_row_group;
   a.sw = w->d_sw;
   a.wsum = w->d_wsum;
   a.bias = (const __half*)bias;
-  a.Y = (__half*)Y;
-  a.ldy = ldy;
   a.w_packed = (const uint8_t*)w->d_w;
   for (int k = 0; k < g->G; ++k) {
     a.seg_end[k] = w->seg_end[k];
@@ -464,9 +538,17 @@ extern "C" dgq_status dgq_linear(const dgq_groups* g, const dgq_weight* w, int t
   a.n_tiles_m = (int)((M + GEMM_BM - 1) / GEMM_BM);
   a.n_tiles_n = (w->N + BN - 1) / BN;
 
-  CUtensorMap tmA, tmB;
+  CUtensorMap tmA, tmB, tmY;
   std::memset(&tmA, 0, sizeof(tmA));
   std::memset(&tmB, 0, sizeof(tmB));
+  std::memset(&tmY, 0, sizeof(tmY));
+  {  // output: panels of 32 fp16 columns x 128 rows, 64-byte swizzle
+    const uint64_t dims[2] = {(uint64_t)w->N, (uint64_t)M};
+    const uint64_t strides[1] = {(uint64_t)ldy * 2};
+    const uint32_t box[2] = {32u, (uint32_t)GEMM_BM};
+    if (!encode_map(&tmY, Y, 2, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_DATA_TYPE_FLOAT16))
+      return DGQ_ERR_CUDA;
+  }
   if (conv) {
     if (layout != DGQ_CODES_S8_CENTRED || mode != DGQ_MODE_STATIC || g->R != 1) return DGQ_ERR_UNSUPPORTED;
     if (conv->c != g->C || (int64_t)conv->n * conv->h * conv->w != M) return DGQ_ERR_INVALID_ARG;
@@ -485,9 +567,6 @@ extern "C" dgq_status dgq_linear(const dgq_groups* g, const dgq_weight* w, int t
     }
     a.conv_W = conv->w;
     a.conv_H = conv->h;
-    a.box_w = bw;
-    a.box_h = bh;
-    a.box_n = bn;
     const uint64_t Cp = (uint64_t)g->K_pad;
     const uint64_t dims[4] = {Cp, (uint64_t)conv->w, (uint64_t)conv->h, (uint64_t)conv->n};
     const uint64_t strides[3] = {Cp, Cp * conv->w, Cp * conv->w * conv->h};
@@ -511,7 +590,7 @@ extern "C" dgq_status dgq_linear(const dgq_groups* g, const dgq_weight* w, int t
   const int grid = std::min(a.n_tiles_m * a.n_tiles_n, n_sm);
   const bool w4 = (w->w_bits == 4);
   cudaStream_t st = (cudaStream_t)stream;
-  if (BN == 160) return launch_gemm_bn<160>(w4, conv != nullptr, tmA, tmB, a, grid, st);
-  if (BN == 64) return launch_gemm_bn<64>(w4, conv != nullptr, tmA, tmB, a, grid, st);
-  return launch_gemm_bn<128>(w4, conv != nullptr, tmA, tmB, a, grid, st);
+  if (BN == 160) return launch_gemm_bn<160>(w4, conv != nullptr, tmA, tmB, tmY, a, grid, st);
+  if (BN == 64) return launch_gemm_bn<64>(w4, conv != nullptr, tmA, tmB, tmY, a, grid, st);
+  return launch_gemm_bn<128>(w4, conv != nullptr, tmA, tmB, tmY, a, grid, st);
 }

@@ -15,6 +15,8 @@ struct dgq_weight {
   int8_t* d_w = nullptr;         // 8-bit: [N_pad][Kt] s8; 4-bit: [N_pad][Kt/2] packed
   float* d_sw = nullptr;         // [N_pad]; 4-bit: sw / 16 (the unpacked codes carry a factor 16)
   float* d_wsum = nullptr;       // [G][N_pad] column sums per group as fp32 (exact); 4-bit: x 16
+  float* d_wres = nullptr;       // [G][N_pad] part of wsum the padding positions could not absorb
+  uint32_t res_mask = 0;         // bit g set: group g has a non-zero entry in d_wres
 };
 
 namespace dgq {
@@ -59,7 +61,7 @@ static dgq_status weight_build(const dgq_groups* g, const int8_t* wq, const floa
   w->seg_end.resize(g->G);
   // GEMM reduction order: group-major; inside a group tap-major (conv), then the group's padded positions
   std::vector<int8_t> Wp((size_t)w->N_pad * w->Kt, 0);
-  std::vector<float> wsum((size_t)g->G * w->N_pad, 0.f);
+  std::vector<float> wsum((size_t)g->G * w->N_pad, 0.f), wres((size_t)g->G * w->N_pad, 0.f);
   const float unit = (w_bits == 4) ? 16.f : 1.f;
   int pos = 0;
   for (int k = 0; k < g->G; ++k) {
@@ -71,12 +73,27 @@ static dgq_status weight_build(const dgq_groups* g, const int8_t* wq, const floa
         for (int o = 0; o < N; ++o) Wp[(size_t)o * w->Kt + pos] = wq[(size_t)o * K + t * g->C + c];
       }
     w->seg_end[k] = pos / DGQ_K_ATOM;
+    const int seg0 = pos - taps * (p1 - p0);  // first reduction position of this group
     for (int o = 0; o < N; ++o) {
       int64_t sum = 0;
       for (int c = 0; c < g->C; ++c)
         if (g->col_group[c] == k)
           for (int t = 0; t < taps; ++t) sum += wq[(size_t)o * K + t * g->C + c];
       wsum[(size_t)k * w->N_pad + o] = (float)sum * unit;
+      // Linear layers: spread -sum over the group's padding positions (whose activation code is the
+      // zero-point Z), so that acc + Z * (-sum) = acc - Z * wsum comes out of the integer product.
+      // What does not fit in the available positions stays in `wres` for the epilogue.
+      int64_t rem = conv ? 0 : -sum;
+      if (!conv)
+        for (int p = p0; p < p1 && rem != 0; ++p)
+          if (g->perm[p] < 0) {
+            const int64_t v = std::max<int64_t>(-qmax, std::min<int64_t>(qmax, rem));
+            Wp[(size_t)o * w->Kt + seg0 + (p - p0)] = (int8_t)v;
+            rem -= v;
+          }
+      const int64_t res = conv ? sum : -rem;  // conv uses zero-centred codes: no zero-point term at all
+      wres[(size_t)k * w->N_pad + o] = (float)res * unit;
+      if (res != 0 && !conv) w->res_mask |= 1u << k;
     }
   }
   std::vector<float> swp(w->N_pad, 0.f);
@@ -97,10 +114,12 @@ static dgq_status weight_build(const dgq_groups* g, const int8_t* wq, const floa
   }
   up((void**)&w->d_sw, swp.data(), swp.size() * sizeof(float));
   up((void**)&w->d_wsum, wsum.data(), wsum.size() * sizeof(float));
+  up((void**)&w->d_wres, wres.data(), wres.size() * sizeof(float));
   if (st != DGQ_OK) {
     cudaFree(w->d_w);
     cudaFree(w->d_sw);
     cudaFree(w->d_wsum);
+    cudaFree(w->d_wres);
     delete w;
     return st;
   }
@@ -148,6 +167,7 @@ extern "C" dgq_status dgq_weight_destroy(dgq_weight* w) {
   cudaFree(w->d_w);
   cudaFree(w->d_sw);
   cudaFree(w->d_wsum);
+  cudaFree(w->d_wres);
   delete w;
   return DGQ_OK;
 }
