@@ -149,7 +149,8 @@ dgq_status dgq_weight_export(const dgq_weight* w, int8_t* wq, float* sw);
  * zero-padded convolution of the NHWC code tensor as an implicit GEMM; needs
  * the S8_CENTRED layout, STATIC mode and channel-only grouping (R = 1).
  * Errors: INVALID_ARG, ALIGNMENT, NOT_CALIBRATED, UNSUPPORTED (K_pad * 255 * 127
- * would overflow int32; conv shape outside the supported tiling), CUDA. */
+ * would overflow int32; more column blocks of 128-160 outputs than the GPU has SMs;
+ * conv shape outside the supported tiling), CUDA. */
 dgq_status dgq_linear(const dgq_groups* g, const dgq_weight* w, int timestep, int mode, int layout,
                       const void* Xq, const float* dyn_scale, const int32_t* dyn_zp, const void* bias,
                       void* Y, int64_t M, int64_t ldy, const dgq_conv_desc* conv, void* stream);

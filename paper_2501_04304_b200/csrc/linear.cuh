@@ -8,7 +8,8 @@
 //   warps 0-15  epilogue: lane quarter = warp & 3 (the TMEM lanes a warp may read), column slice = warp >> 2
 //   warp  16    TMA producer (one elected lane): A code tile and B weight tile per 128-byte K stage
 //   warp  17    MMA issuer (one elected lane) and TMEM allocator
-//   warps 18-21 (4-bit weights only) unpack packed nibbles from global memory into the B stage
+//   warp  18    output store (one elected lane): TMA stores of the staged fp16 tile
+//   warps 19-21 (4-bit weights only) unpack packed nibbles from global memory into the B stage
 // K runs over 32-code atoms; a stage holds four atoms.  Group segments are multiples of one atom,
 // so the issuer moves to the next TMEM accumulator between two atoms, commits the finished one to
 // the epilogue and keeps going while the epilogue drains it.
@@ -21,7 +22,9 @@
 // wsum (flagged in `res_mask`).
 //
 // Output: the fp16 tile is staged in shared memory in 64-byte-swizzled panels of 32 columns and
-// written with TMA stores, which also clip the ragged last row and column tiles.
+// written with TMA stores, which also clip the ragged last row and column tiles.  The epilogue
+// warps only signal "staged" and move on to the next tile; the store warp issues the stores and
+// signals "staging free" once they have read the buffer.
 // Linear layers: A and B stages are 128-byte-swizzled tiles fetched with one TMA box each.
 // 3x3 conv (implicit GEMM): the reduction order is group-major, then filter tap, then channel
 // atom; every A atom is its own 32-byte-swizzled 4-D TMA box of the NHWC code tensor shifted by
@@ -37,8 +40,11 @@ constexpr int GEMM_EPI_WARPS = 16;
 constexpr int GEMM_EPI_THREADS = GEMM_EPI_WARPS * 32;
 constexpr int GEMM_WARP_TMA = 16;
 constexpr int GEMM_WARP_MMA = 17;
-constexpr int GEMM_THREADS_W8 = 18 * 32;
-constexpr int GEMM_THREADS_W4 = 22 * 32;
+constexpr int GEMM_WARP_STORE = 18;
+constexpr int GEMM_THREADS_W8 = 19 * 32;
+constexpr int GEMM_UNPACK_WARPS = 3;
+constexpr int GEMM_UNPACK_THREADS = GEMM_UNPACK_WARPS * 32;
+constexpr int GEMM_THREADS_W4 = GEMM_THREADS_W8 + GEMM_UNPACK_THREADS;
 constexpr int GEMM_A_STAGE = GEMM_BM * 128;  // bytes
 constexpr int GEMM_SMEM_LIMIT = 227 * 1024;
 
@@ -47,7 +53,7 @@ struct GemmCfg {
   static constexpr int B_STAGE = BN * 128;
   static constexpr int STAGE = GEMM_A_STAGE + B_STAGE;
   static constexpr int OUT_BYTES = GEMM_BM * BN * 2;  // fp16 staging of one output tile
-  static constexpr int MISC_BYTES = 2048 + BN * 8;    // barriers + sw / bias of the tile's columns
+  static constexpr int MISC_BYTES = 2048 + (2 + DGQ_MAX_GROUPS) * BN * 4;  // barriers + sw, bias, wsum of the CTA's columns
   static constexpr int STAGES_RAW = (GEMM_SMEM_LIMIT - 1024 - OUT_BYTES - MISC_BYTES) / STAGE;
   static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
   static constexpr int NACC_RAW = 512 / BN;
@@ -89,19 +95,11 @@ struct __align__(8) GemmShared {
   uint64_t empty[8];
   uint64_t acc_full[4];
   uint64_t acc_empty[4];
-  uint64_t epi_bar;
+  uint64_t out_full;   // all epilogue warps have staged their part of the output tile
+  uint64_t out_free;   // the TMA stores of the previous tile have read the staging buffer
   uint32_t tmem_base;
   int abort_flag;
 };
-
-// Barrier among the epilogue warps with a bounded wait (one arrival per warp).
-__device__ __forceinline__ bool epi_sync(uint64_t* bar, uint32_t& phase, int lane, volatile int* abort_flag) {
-  __syncwarp();
-  if (lane == 0) mbar_arrive(bar);
-  const bool ok = __all_sync(0xffffffffu, mbar_wait(bar, phase & 1u, abort_flag));
-  phase ^= 1u;
-  return ok;
-}
 
 template <int BN, bool W4, bool CONV>
 __global__ void __launch_bounds__(W4 ? GEMM_THREADS_W4 : GEMM_THREADS_W8, 1)
@@ -117,8 +115,12 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   unsigned char* smB = smem + STAGES * GEMM_A_STAGE;
   unsigned char* smOut = smem + STAGES * Cfg::STAGE;  // 1024-byte aligned: every stage size is
   GemmShared* sh = reinterpret_cast<GemmShared*>(smOut + Cfg::OUT_BYTES);
-  float* sw_s = reinterpret_cast<float*>(smOut + Cfg::OUT_BYTES + 2048);
-  float* bias_s = sw_s + BN;
+  // Every tile of this CTA has the same column block (the grid is a multiple of the number of
+  // column blocks), so its per-column constants are loaded once.
+  float* sw_s = reinterpret_cast<float*>(smOut + Cfg::OUT_BYTES + 2048);  // [BN]
+  float* bias_s = sw_s + BN;                                              // [BN]
+  float* wsum_s = bias_s + BN;                                            // [G][BN]
+  const int cta_n0 = ((int)blockIdx.x % a.n_tiles_n) * BN;
   volatile int* abort_flag = &sh->abort_flag;
 
   const int warp = threadIdx.x >> 5;
@@ -129,17 +131,28 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) {
-      mbar_init(&sh->full[i], W4 ? 5 : 1);
+      mbar_init(&sh->full[i], W4 ? 1 + GEMM_UNPACK_WARPS : 1);
       mbar_init(&sh->empty[i], 1);
     }
     for (int i = 0; i < NACC; ++i) {
       mbar_init(&sh->acc_full[i], 1);
       mbar_init(&sh->acc_empty[i], GEMM_EPI_WARPS);
     }
-    mbar_init(&sh->epi_bar, GEMM_EPI_WARPS);
+    mbar_init(&sh->out_full, GEMM_EPI_WARPS);
+    mbar_init(&sh->out_free, 1);
     sh->abort_flag = 0;
     fence_barrier_init();
   }
+  for (int i = threadIdx.x; i < BN; i += blockDim.x) {
+    const int col = cta_n0 + i;
+    sw_s[i] = col < a.N_pad ? __ldg(a.sw + col) : 0.f;
+    bias_s[i] = (a.bias != nullptr && col < a.N) ? __half2float(a.bias[col]) : 0.f;
+  }
+  if (a.use_zp)
+    for (int i = threadIdx.x; i < a.G * BN; i += blockDim.x) {
+      const int g = i / BN, c = i - g * BN;
+      wsum_s[i] = cta_n0 + c < a.N_pad ? __ldg(a.wsum + (size_t)g * a.N_pad + cta_n0 + c) : 0.f;
+    }
   if (warp == GEMM_WARP_MMA) {
     tmem_alloc(&sh->tmem_base, 512);
     tmem_relinquish();
@@ -154,7 +167,6 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (lane == 0) {
       tma_prefetch_desc(&tmA);
       if (!W4) tma_prefetch_desc(&tmB);
-      tma_prefetch_desc(&tmY);
       uint32_t it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
@@ -206,11 +218,8 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         int g = 0;
-        bool first = true;
-        int ab = acc_it % NACC;
-        ok = mbar_wait(&sh->acc_empty[ab], ((acc_it / NACC) & 1) ^ 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
+        bool need_acc = true;  // the next atom starts a group: take the next accumulator first
+        int ab = 0;
         for (int ks = 0; ks < n_kstages && ok; ++ks, ++it) {
           const int s = it % STAGES;
           ok = mbar_wait(&sh->full[s], (it / STAGES) & 1, abort_flag);
@@ -221,11 +230,7 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const uint32_t b_addr = smem_u32(smB + s * Cfg::B_STAGE);
           for (int j = 0; j < atoms_here && ok; ++j) {
             const int atom = ks * 4 + j;
-            if (atom >= a.seg_end[g]) {  // group finished: hand its accumulator to the epilogue
-              mma_commit(&sh->acc_full[ab]);
-              ++acc_it;
-              ++g;
-              first = true;
+            if (need_acc) {
               ab = acc_it % NACC;
               ok = mbar_wait(&sh->acc_empty[ab], ((acc_it / NACC) & 1) ^ 1, abort_flag);
               if (!ok) break;
@@ -233,14 +238,16 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             const uint64_t da = CONV ? smem_desc(a_addr + j * 4096, 256, 6) : smem_desc(a_addr + j * 32, 1024, 2);
             const uint64_t db = smem_desc(b_addr + j * 32, 1024, 2);
-            mma_i8(tmem_base + (uint32_t)(ab * BN), da, db, a.idesc, first ? 0u : 1u);
-            first = false;
+            mma_i8(tmem_base + (uint32_t)(ab * BN), da, db, a.idesc, need_acc ? 0u : 1u);
+            need_acc = false;
+            if (atom + 1 == a.seg_end[g]) {  // last atom of the group: hand the accumulator over right away
+              mma_commit(&sh->acc_full[ab]);
+              ++acc_it;
+              ++g;
+              need_acc = true;
+            }
           }
           if (ok) mma_commit(&sh->empty[s]);  // stage reusable once these MMAs have read it
-        }
-        if (ok) {
-          mma_commit(&sh->acc_full[ab]);
-          ++acc_it;
         }
       }
     }
@@ -250,107 +257,139 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     constexpr int NCH = CW / 8;
     const int q = warp & 3, sl = warp >> 2;
     const int r_tile = q * 32 + lane;  // row inside the tile = TMEM lane
-    uint32_t acc_it = 0, sync_phase = 0;
+    uint32_t acc_it = 0, tile_it = 0;
     bool ok = true;
-    bool stored = false;
-    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-      const int tm = tile / a.n_tiles_n, tn = tile - tm * a.n_tiles_n;
-      const int n0 = tn * BN;
+    // The first scale / zero-point of the row are fetched one tile ahead, so their latency hides
+    // behind the current tile.
+    float pre_s = 0.f;
+    int pre_z = 0;
+    const float* srow = nullptr;
+    const int32_t* zrow = nullptr;
+    auto prefetch_tile = [&](int tile) {
+      const int tm = tile / a.n_tiles_n;
       const int64_t row = (int64_t)tm * GEMM_BM + r_tile;
       const int64_t row_c = row < a.M ? row : a.M - 1;
-      const int col0 = n0 + sl * CW;
-      const int64_t prow = a.per_token ? row_c : (int64_t)a.row_group[row_c % a.P];
-      const float* srow = a.scale + prow * a.G;
-      const int32_t* zrow = a.zp + prow * a.G;
-      // per-column constants of this tile (read again only after the next barrier)
-      for (int i = threadIdx.x; i < BN; i += GEMM_EPI_THREADS) {
-        const int col = n0 + i;
-        sw_s[i] = col < a.N_pad ? __ldg(a.sw + col) : 0.f;
-        bias_s[i] = (a.bias != nullptr && col < a.N) ? __half2float(a.bias[col]) : 0.f;
-      }
+      const int64_t prow = a.per_token ? row_c : (int64_t)__ldg(a.row_group + row_c % a.P);
+      srow = a.scale + prow * a.G;
+      zrow = a.zp + prow * a.G;
+      pre_s = __ldg(srow);
+      pre_z = a.use_zp ? __ldg(zrow) : 0;
+    };
+    if ((int)blockIdx.x < n_tiles) prefetch_tile(blockIdx.x);
+    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tile_it) {
+      const int col0 = cta_n0 + sl * CW;
+      const float* srow_t = srow;
+      const int32_t* zrow_t = zrow;
       float y[CW];
 #pragma unroll
       for (int i = 0; i < CW; ++i) y[i] = 0.f;
-      float s_next = __ldg(srow);
+      // scale and zero-point of the next group are fetched one group ahead
+      float s_next = pre_s;
+      int z_next = pre_z;
       for (int g = 0; g < a.G && ok; ++g, ++acc_it) {
         const float s = s_next;
-        if (g + 1 < a.G) s_next = __ldg(srow + g + 1);
-        float c1 = 0.f, c2 = 0.f;
-        if (a.use_zp) {
-          const int Z = __ldg(zrow + g);
-          const int Zc = min(max(Z, 0), a.code_max);
-          c1 = -s * (float)(Z - Zc);
-          c2 = ((a.res_mask >> g) & 1u) ? -s * (float)Zc : 0.f;
+        const int Z = z_next;
+        if (g + 1 < a.G) {
+          s_next = __ldg(srow_t + g + 1);
+          if (a.use_zp) z_next = __ldg(zrow_t + g + 1);
+        } else if (tile + (int)gridDim.x < n_tiles) {
+          prefetch_tile(tile + gridDim.x);
         }
         const int ab = acc_it % NACC;
         ok = __all_sync(0xffffffffu, mbar_wait(&sh->acc_full[ab], (acc_it / NACC) & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * BN + sl * CW);
-        // Two register buffers: the load of chunk k + 1 is in flight while chunk k is converted and
-        // accumulated.  The accumulator is handed back as soon as its last chunk is in registers.
-        uint32_t rb[2][8];
-        tmem_ld8(taddr, rb[0]);
+        // All loads of the group are issued before the single wait, so their latencies overlap; the
+        // accumulator is handed back as soon as its columns are in registers.
+        uint32_t rb[NCH][8];
 #pragma unroll
-        for (int k = 0; k < NCH; ++k) {
-          tmem_ld_wait();
-          if (k + 1 < NCH) {
-            tmem_ld8(taddr + (k + 1) * 8, rb[(k + 1) & 1]);
-          } else {
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sh->acc_empty[ab]);
+        for (int k = 0; k < NCH; ++k) tmem_ld8(taddr + k * 8, rb[k]);
+        tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh->acc_empty[ab]);
+#pragma unroll
+        for (int k = 0; k < NCH; ++k)
+#pragma unroll
+          for (int i = 0; i < 8; ++i) y[k * 8 + i] = fmaf(s, (float)(int)rb[k][i], y[k * 8 + i]);
+        if (a.use_zp) {
+          // rare: Z outside the code range (the stored padding code is the clamped Z), or a group
+          // whose padding could not absorb all of wsum
+          const int Zc = min(max(Z, 0), a.code_max);
+          const float c1 = -s * (float)(Z - Zc);
+          const float c2 = ((a.res_mask >> g) & 1u) ? -s * (float)Zc : 0.f;
+          if (__any_sync(0xffffffffu, c1 != 0.f)) {
+            const float4* ws = reinterpret_cast<const float4*>(wsum_s + g * BN + sl * CW);
+#pragma unroll
+            for (int i = 0; i < CW; i += 4) {
+              const float4 u = ws[i >> 2];
+              y[i] = fmaf(c1, u.x, y[i]);
+              y[i + 1] = fmaf(c1, u.y, y[i + 1]);
+              y[i + 2] = fmaf(c1, u.z, y[i + 2]);
+              y[i + 3] = fmaf(c1, u.w, y[i + 3]);
+            }
           }
+          if ((a.res_mask >> g) & 1u) {
+            const float4* wr = reinterpret_cast<const float4*>(a.wres + (size_t)g * a.N_pad + col0);
 #pragma unroll
-          for (int i = 0; i < 8; ++i) y[k * 8 + i] = fmaf(s, (float)(int)rb[k & 1][i], y[k * 8 + i]);
-        }
-        if (__any_sync(0xffffffffu, c1 != 0.f || c2 != 0.f)) {
-          const float4* ws = reinterpret_cast<const float4*>(a.wsum + (size_t)g * a.N_pad + col0);
-          const float4* wr = reinterpret_cast<const float4*>(a.wres + (size_t)g * a.N_pad + col0);
-#pragma unroll
-          for (int i = 0; i < CW; i += 4) {
-            const float4 u = __ldg(ws + (i >> 2)), v = __ldg(wr + (i >> 2));
-            y[i] = fmaf(c1, u.x, fmaf(c2, v.x, y[i]));
-            y[i + 1] = fmaf(c1, u.y, fmaf(c2, v.y, y[i + 1]));
-            y[i + 2] = fmaf(c1, u.z, fmaf(c2, v.z, y[i + 2]));
-            y[i + 3] = fmaf(c1, u.w, fmaf(c2, v.w, y[i + 3]));
+            for (int i = 0; i < CW; i += 4) {
+              const float4 v = __ldg(wr + (i >> 2));
+              y[i] = fmaf(c2, v.x, y[i]);
+              y[i + 1] = fmaf(c2, v.y, y[i + 1]);
+              y[i + 2] = fmaf(c2, v.z, y[i + 2]);
+              y[i + 3] = fmaf(c2, v.w, y[i + 3]);
+            }
           }
         }
       }
       if (!ok) break;
-      // the previous tile's TMA stores must have finished reading the staging buffer
-      if (stored && threadIdx.x == 0) bulk_wait_read0();
-      ok = epi_sync(&sh->epi_bar, sync_phase, lane, abort_flag);
+      // staging buffer: wait until the stores of the previous tile have read it (normally long done)
+      ok = __all_sync(0xffffffffu, mbar_wait(&sh->out_free, (tile_it & 1) ^ 1, abort_flag));
       if (!ok) break;
 #pragma unroll
       for (int j = 0; j < NCH; ++j) {
         const int cl = sl * CW + j * 8;  // first tile column of this 16-byte chunk
+        const float4 s0 = *reinterpret_cast<const float4*>(sw_s + cl), s1 = *reinterpret_cast<const float4*>(sw_s + cl + 4);
+        const float4 b0 = *reinterpret_cast<const float4*>(bias_s + cl), b1 = *reinterpret_cast<const float4*>(bias_s + cl + 4);
         uint4 o;
         __half2* oh = reinterpret_cast<__half2*>(&o);
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-          oh[k] = __floats2half2_rn(fmaf(sw_s[cl + 2 * k], y[j * 8 + 2 * k], bias_s[cl + 2 * k]),
-                                    fmaf(sw_s[cl + 2 * k + 1], y[j * 8 + 2 * k + 1], bias_s[cl + 2 * k + 1]));
+        oh[0] = __floats2half2_rn(fmaf(s0.x, y[j * 8 + 0], b0.x), fmaf(s0.y, y[j * 8 + 1], b0.y));
+        oh[1] = __floats2half2_rn(fmaf(s0.z, y[j * 8 + 2], b0.z), fmaf(s0.w, y[j * 8 + 3], b0.w));
+        oh[2] = __floats2half2_rn(fmaf(s1.x, y[j * 8 + 4], b1.x), fmaf(s1.y, y[j * 8 + 5], b1.y));
+        oh[3] = __floats2half2_rn(fmaf(s1.z, y[j * 8 + 6], b1.z), fmaf(s1.w, y[j * 8 + 7], b1.w));
         // panel of 32 columns = 64-byte rows, 16-byte chunk index XOR bits 1-2 of the row (64 B swizzle)
         const int panel = cl >> 5, ch = (cl >> 3) & 3;
         *reinterpret_cast<uint4*>(smOut + panel * (GEMM_BM * 64) + r_tile * 64 + ((ch ^ ((r_tile >> 1) & 3)) << 4)) = o;
       }
       fence_proxy_async_smem();
-      ok = epi_sync(&sh->epi_bar, sync_phase, lane, abort_flag);
-      if (!ok) break;
-      if (threadIdx.x == 0) {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh->out_full);
+    }
+  } else if (warp == GEMM_WARP_STORE) {
+    // ------------------------------------------------------------ output store
+    if (lane == 0) {
+      tma_prefetch_desc(&tmY);
+      uint32_t tile_it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tile_it) {
+        const int tm = tile / a.n_tiles_n, tn = tile - tm * a.n_tiles_n;
+        const int n0 = tn * BN;
+        ok = mbar_wait(&sh->out_full, tile_it & 1, abort_flag);
+        if (!ok) break;
 #pragma unroll
         for (int pnl = 0; pnl < BN / 32; ++pnl)
           if (n0 + pnl * 32 < a.N) tma_store_2d(&tmY, smOut + pnl * (GEMM_BM * 64), n0 + pnl * 32, tm * GEMM_BM);
         bulk_commit();
+        bulk_wait_read0();
+        mbar_arrive(&sh->out_free);
       }
-      stored = true;
+      bulk_wait0();
     }
-    if (stored && threadIdx.x == 0) bulk_wait0();
   } else if (W4) {
     // ------------------------------------------------------------ 4-bit weight unpack into the B stage
-    constexpr int ITEMS = BN * 4 / 128;  // 16-byte packed pieces per thread and stage
-    const int ut = threadIdx.x - GEMM_THREADS_W8;  // 0..127
+    constexpr int ITEMS = (BN * 4 + GEMM_UNPACK_THREADS - 1) / GEMM_UNPACK_THREADS;  // 16-byte pieces per thread
+    const int ut = threadIdx.x - GEMM_THREADS_W8;  // 0..GEMM_UNPACK_THREADS-1
     uint32_t it = 0;
     bool ok = true;
     const int row_bytes = a.Kt >> 1;
@@ -359,11 +398,11 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int n0 = (tile % a.n_tiles_n) * BN;
 #pragma unroll
       for (int e = 0; e < ITEMS; ++e) {
-        const int item = ut + e * 128;
+        const int item = ut + e * GEMM_UNPACK_THREADS;
         const int r = item >> 2, qd = item & 3;  // B row, 16-byte packed quarter of the 64-byte row slice
         const int kb = ks * 64 + qd * 16;
         pk[e] = make_uint4(0u, 0u, 0u, 0u);
-        if (kb < row_bytes)
+        if (item < BN * 4 && kb < row_bytes)
           pk[e] = __ldg(reinterpret_cast<const uint4*>(a.w_packed + (size_t)(n0 + r) * row_bytes + kb));
       }
     };
@@ -376,7 +415,8 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         unsigned char* bst = smB + s * Cfg::B_STAGE;
 #pragma unroll
         for (int e = 0; e < ITEMS; ++e) {
-          const int item = ut + e * 128;
+          const int item = ut + e * GEMM_UNPACK_THREADS;
+          if (item >= BN * 4) continue;
           const int r = item >> 2, qd = item & 3;
           const uint4 p4 = pk[e];
           const uint4 c0 = make_uint4((p4.x << 4) & 0xF0F0F0F0u, p4.x & 0xF0F0F0F0u, (p4.y << 4) & 0xF0F0F0F0u,
@@ -587,7 +627,9 @@ extern "C" dgq_status dgq_linear(const dgq_groups* g, const dgq_weight* w, int t
   int dev = 0, n_sm = 148;
   DGQ_CUDA_OK(cudaGetDevice(&dev));
   DGQ_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
-  const int grid = std::min(a.n_tiles_m * a.n_tiles_n, n_sm);
+  // a multiple of the number of column blocks, so that every CTA keeps one column block
+  if (a.n_tiles_n > n_sm) return DGQ_ERR_UNSUPPORTED;
+  const int grid = std::min(a.n_tiles_m, n_sm / a.n_tiles_n) * a.n_tiles_n;
   const bool w4 = (w->w_bits == 4);
   cudaStream_t st = (cudaStream_t)stream;
   if (BN == 160) return launch_gemm_bn<160>(w4, conv != nullptr, tmA, tmB, tmY, a, grid, st);
