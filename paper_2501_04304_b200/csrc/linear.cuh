@@ -72,6 +72,7 @@ struct GemmArgs {
   int n_tiles_m, n_tiles_n;
   uint32_t idesc;
   int use_zp;                 // 0 for zero-centred codes
+  int magic;                  // 1: |acc| < 2^22 for every group, the epilogue converts without I2F
   int code_max;               // 2^b - 1
   uint32_t res_mask;          // groups whose padding did not absorb all of wsum
   int per_token;              // 1: scale rows indexed by token, 0: by row_group[token mod P]
@@ -101,7 +102,7 @@ struct __align__(8) GemmShared {
   int abort_flag;
 };
 
-template <int BN, bool W4, bool CONV>
+template <int BN, bool W4, bool CONV, bool MAGIC>
 __global__ void __launch_bounds__(W4 ? GEMM_THREADS_W4 : GEMM_THREADS_W8, 1)
 gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmY, const __grid_constant__ GemmArgs a) {
@@ -309,10 +310,23 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh->acc_empty[ab]);
+        if (MAGIC) {
+          // |acc| < 2^22: adding 0x4B400000 gives the bit pattern of the float 1.5 * 2^23 + acc, and
+          // subtracting 1.5 * 2^23 is exact.  Integer add and float add are full-rate instructions;
+          // the int -> float conversion runs on the 16-lane special-function pipe and would bound
+          // the whole kernel.
 #pragma unroll
-        for (int k = 0; k < NCH; ++k)
+          for (int k = 0; k < NCH; ++k)
 #pragma unroll
-          for (int i = 0; i < 8; ++i) y[k * 8 + i] = fmaf(s, (float)(int)rb[k][i], y[k * 8 + i]);
+            for (int i = 0; i < 8; ++i)
+              y[k * 8 + i] =
+                  fmaf(s, __fsub_rn(__int_as_float((int)rb[k][i] + 0x4B400000), 12582912.0f), y[k * 8 + i]);
+        } else {
+#pragma unroll
+          for (int k = 0; k < NCH; ++k)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) y[k * 8 + i] = fmaf(s, (float)(int)rb[k][i], y[k * 8 + i]);
+        }
         if (a.use_zp) {
           // rare: Z outside the code range (the stored padding code is the clamped Z), or a group
           // whose padding could not absorb all of wsum
@@ -491,7 +505,7 @@ static bool encode_map(CUtensorMap* m, const void* base, int rank, const uint64_
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, bool W4, bool CONV>
+template <int BN, bool W4, bool CONV, bool MAGIC>
 static dgq_status launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
                               const GemmArgs& a, int grid, cudaStream_t stream) {
   using Cfg = GemmCfg<BN>;
@@ -499,11 +513,11 @@ static dgq_status launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, co
   int dev = 0;
   DGQ_CUDA_OK(cudaGetDevice(&dev));
   if (dev >= 64 || !attr_set[dev]) {
-    DGQ_CUDA_OK(cudaFuncSetAttribute(gq_gemm_kernel<BN, W4, CONV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    DGQ_CUDA_OK(cudaFuncSetAttribute(gq_gemm_kernel<BN, W4, CONV, MAGIC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      Cfg::SMEM));
     if (dev < 64) attr_set[dev] = true;
   }
-  gq_gemm_kernel<BN, W4, CONV><<<grid, W4 ? GEMM_THREADS_W4 : GEMM_THREADS_W8, Cfg::SMEM, stream>>>(tmA, tmB, tmY, a);
+  gq_gemm_kernel<BN, W4, CONV, MAGIC><<<grid, W4 ? GEMM_THREADS_W4 : GEMM_THREADS_W8, Cfg::SMEM, stream>>>(tmA, tmB, tmY, a);
   g_launches += 1;
   DGQ_CUDA_OK(cudaGetLastError());
   return DGQ_OK;
@@ -512,11 +526,18 @@ static dgq_status launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, co
 template <int BN>
 static dgq_status launch_gemm_bn(bool w4, bool conv, const CUtensorMap& tmA, const CUtensorMap& tmB,
                                  const CUtensorMap& tmY, const GemmArgs& a, int grid, cudaStream_t stream) {
+  if (a.magic) {
+    if (w4)
+      return conv ? launch_gemm<BN, true, true, true>(tmA, tmB, tmY, a, grid, stream)
+                  : launch_gemm<BN, true, false, true>(tmA, tmB, tmY, a, grid, stream);
+    return conv ? launch_gemm<BN, false, true, true>(tmA, tmB, tmY, a, grid, stream)
+                : launch_gemm<BN, false, false, true>(tmA, tmB, tmY, a, grid, stream);
+  }
   if (w4)
-    return conv ? launch_gemm<BN, true, true>(tmA, tmB, tmY, a, grid, stream)
-                : launch_gemm<BN, true, false>(tmA, tmB, tmY, a, grid, stream);
-  return conv ? launch_gemm<BN, false, true>(tmA, tmB, tmY, a, grid, stream)
-              : launch_gemm<BN, false, false>(tmA, tmB, tmY, a, grid, stream);
+    return conv ? launch_gemm<BN, true, true, false>(tmA, tmB, tmY, a, grid, stream)
+                : launch_gemm<BN, true, false, false>(tmA, tmB, tmY, a, grid, stream);
+  return conv ? launch_gemm<BN, false, true, false>(tmA, tmB, tmY, a, grid, stream)
+              : launch_gemm<BN, false, false, false>(tmA, tmB, tmY, a, grid, stream);
 }
 
 }  // namespace dgq
@@ -567,6 +588,17 @@ extern "C" dgq_status dgq_linear(const dgq_groups* g, const dgq_weight* w, int t
     a.seg_end[k] = w->seg_end[k];
     a.grp_atoms[k] = (g->group_off[k + 1] - g->group_off[k]) / DGQ_K_ATOM;
     a.grp_chan0[k] = g->group_off[k];
+  }
+  {
+    // |acc| < 2^22 holds for a group of n atoms if n * 32 * max|code| * max|weight| < 2^22
+    const int64_t amax = (layout == DGQ_CODES_S8_CENTRED) ? 128 : (1 << g->bits) - 1;
+    const int64_t wmax = (w->w_bits == 4) ? 7 * 16 : 127;
+    int longest = 0, start = 0;
+    for (int k = 0; k < g->G; ++k) {
+      longest = std::max(longest, w->seg_end[k] - start);
+      start = w->seg_end[k];
+    }
+    a.magic = (longest * (int64_t)DGQ_K_ATOM * amax * wmax < (1ll << 22)) ? 1 : 0;
   }
   int BN = 128;
   if (w->N % 160 == 0) BN = 160;
