@@ -166,43 +166,65 @@ class Workload:
             tot += v.numel() * v.element_size()
         return tot
 
-    def step(self, i, timers=None):
-        """All kernels of one step on buffer set i.  `timers` collects (kind, start, stop) CUDA events."""
-        b, torch = self.b, self.torch
+    KINDS = ("quantize", "gemm", "attention")
+
+    def launch_kind(self, kind, i):
+        """Enqueues the kernels of one kind of one step on buffer set i (order of a step: every
+        activation quantizer, then every GEMM and the conv, then the cross-attention)."""
+        b = self.b
         s = self.sets[i % self.n_sets]
+        if kind == "quantize":
+            for key in INPUT_C:
+                b.quantize_act_into(self.groups[key], s["in"][key], s["codes"][key], s["ds"][key], s["dz"][key],
+                                    mode=b.MODE_DYNAMIC_TOKEN)
+            b.quantize_act_into(self.conv_groups, s["in"]["conv"], s["conv_codes"], None, None,
+                                layout=b.CODES_S8_CENTRED)
+        elif kind == "gemm":
+            for name, N, K, key in LINEARS:
+                b.linear(self.groups[key], self.weights[name], s["codes"][key], mode=b.MODE_DYNAMIC_TOKEN,
+                         dyn_scale=s["ds"][key], dyn_zp=s["dz"][key], bias=self.biases[name], out=s["out"][name])
+            b.linear(self.conv_groups, self.conv_weight, s["conv_codes"], layout=b.CODES_S8_CENTRED,
+                     bias=self.conv_bias, out=s["conv_out"], conv=self.conv_desc)
+        else:
+            b.cross_attn_logq(s["in"]["Q"], s["in"]["K"], s["in"]["V"], ATT["bits"], out=s["attn_out"],
+                              workspace=s["attn_ws"])
 
-        def timed(kind, fn):
-            if timers is None:
-                fn()
-                return
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            fn()
-            e1.record()
-            timers.append((kind, e0, e1))
+    def step(self, i):
+        for kind in self.KINDS:
+            self.launch_kind(kind, i)
 
-        for key in INPUT_C:
-            timed("quantize", lambda key=key: b.quantize_act_into(
-                self.groups[key], s["in"][key], s["codes"][key], s["ds"][key], s["dz"][key],
-                mode=b.MODE_DYNAMIC_TOKEN))
-        for name, N, K, key in LINEARS:
-            timed("gemm", lambda name=name, key=key: b.linear(
-                self.groups[key], self.weights[name], s["codes"][key], mode=b.MODE_DYNAMIC_TOKEN,
-                dyn_scale=s["ds"][key], dyn_zp=s["dz"][key], bias=self.biases[name], out=s["out"][name]))
-        timed("attention", lambda: b.cross_attn_logq(s["in"]["Q"], s["in"]["K"], s["in"]["V"], ATT["bits"],
-                                                     out=s["attn_out"], workspace=s["attn_ws"]))
-        timed("quantize", lambda: b.quantize_act_into(self.conv_groups, s["in"]["conv"], s["conv_codes"], None, None,
-                                                      layout=b.CODES_S8_CENTRED))
-        timed("gemm", lambda: b.linear(self.conv_groups, self.conv_weight, s["conv_codes"],
-                                       layout=b.CODES_S8_CENTRED, bias=self.conv_bias, out=s["conv_out"],
-                                       conv=self.conv_desc))
+    def capture(self):
+        """One CUDA graph per (buffer set, kind): launch overhead stays out of the timed region."""
+        torch = self.torch
+        self.graphs, self.stream = [], torch.cuda.Stream()
+        n0 = self.b.launch_count()
+        with torch.cuda.stream(self.stream):
+            for i in range(self.n_sets):
+                gs = {}
+                for kind in self.KINDS:
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=self.stream):
+                        self.launch_kind(kind, i)
+                    gs[kind] = g
+                self.graphs.append(gs)
+        torch.cuda.synchronize()
+        self.launches_per_step = (self.b.launch_count() - n0) // self.n_sets
+
+    def replay_step(self, i, marks=None):
+        gs = self.graphs[i % self.n_sets]
+        for kind in self.KINDS:
+            if marks is not None:
+                e = self.torch.cuda.Event(enable_timing=True)
+                e.record()
+                marks.append((kind, e))
+            gs[kind].replay()
 
     def step_e2e(self, i):
         """The same step through host buffers: inputs copied from pinned memory, results read back."""
         s = self.sets[i % self.n_sets]
         for k, h in self.host.items():
             s["in"][k].copy_(h, non_blocking=True)
-        self.step(i)
+        self.replay_step(i)
         self.host_out["ff2"].copy_(s["out"]["ff2"], non_blocking=True)
         self.host_out["conv"].copy_(s["conv_out"], non_blocking=True)
         self.host_out["attn"].copy_(s["attn_out"], non_blocking=True)
@@ -239,21 +261,24 @@ def run_cuda(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(max(args.warmup, 3)):
+    for i in range(3):
         wl.step(i)
+    barrier()
+    wl.capture()
+    for i in range(max(args.warmup, 3)):
+        wl.replay_step(i)
     barrier()
     sampler = ClockSampler(local)
     sampler.start()
-    timers = []
-    launches0 = b.launch_count()
+    marks = []
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record()
     for i in range(args.steps):
-        wl.step(i, timers)
+        wl.replay_step(i, marks)
     e1.record()
     barrier()
-    launches = b.launch_count() - launches0
+    launches = wl.launches_per_step * args.steps
     ms_total = e0.elapsed_time(e1)
     # end to end: host buffers in, results out, every step
     for i in range(2):
@@ -271,9 +296,11 @@ def run_cuda(args):
     if status != 0:
         raise RuntimeError(f"a kernel recorded status {status} ({b.status_string(status)})")
 
+    # duration of a kind = from its mark to the next mark (or to the end of the timed region)
     kind_ms = {}
-    for kind, a0, a1 in timers:
-        kind_ms.setdefault(kind, []).append(a0.elapsed_time(a1))
+    for j, (kind, ev) in enumerate(marks):
+        nxt = marks[j + 1][1] if j + 1 < len(marks) else e1
+        kind_ms.setdefault(kind, []).append(ev.elapsed_time(nxt))
     t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -302,7 +329,7 @@ def run_cuda(args):
         "gpu_launches": int(launches),
         "roofline": {"bound": "tensor", "achieved": gemm_tops, "peak": int8_peak, "unit": "TOP/s",
                      "frac": gemm_tops / int8_peak, "traffic": None,
-                     "kernel": "gq_gemm_kernel (8 launches per step)",
+                     "kernel": "gq_gemm_kernel (8 launches per step, timed as one CUDA graph)",
                      "peak_source": f"2 x bf16 sustained, {peaks['source']}"},
         "kernels": {
             "gemm": {"ms_per_step": gemm_ms, "tops": gemm_tops, "frac_int8_peak": gemm_tops / int8_peak},
