@@ -7,19 +7,40 @@
 //            off-<start> log2-score of the scope, reduced with an ordered-integer atomicMax;
 //   phase 2  the same logits again (bit-identical), codes in the log domain
 //            code = clamp(rint(log2 s - log2 A_ij), 0, 2^b - 1) with no transcendental per score,
-//            2^-code built by writing the fp16 exponent field, A_hat V on tensor cores, and the
+//            2^-code built by writing the exponent field, A_hat V on tensor cores, and the
 //            <start> column added as a separate fp32 rank-1 term A_i0 V_0.
-// One CTA = one (prompt, head, 128 query rows); 8 warps of 16 rows.  K and V^T of the head sit in
-// shared memory.  HBM traffic: Q and O once (the second read of Q is served by L2), K and V once.
+// One CTA = one (prompt, head, block of query rows); 8 warps, each owning 16 or 32 rows.  K and
+// V^T of the head sit in shared memory (column 0 of V^T zeroed: the <start> key never enters the
+// quantized product).  Every warp stages its Q rows in shared memory with coalesced 128-bit loads
+// and writes its O rows back the same way.  HBM traffic: Q and O once (the second read of Q is
+// served by L2), K and V once per CTA from L2.
 #pragma once
 
 #include "common.cuh"
 
 namespace dgq {
 
-constexpr int AT_ROWS = 128;
-constexpr int AT_THREADS = 256;
+constexpr int AT_WARPS = 8;
+constexpr int AT_THREADS = AT_WARPS * 32;
 constexpr float AT_P_SHIFT = 14.0f;  // A_hat / s is held in fp16 as 2^(14 - code)
+constexpr float AT_CODE_CAP = 40.0f; // 2^(14 - 40) is below half the smallest fp16: codes beyond it give 0
+
+template <int D, int NKP>
+struct AttnCfg {
+  static constexpr int DP = (D + 15) / 16 * 16;   // features padded to the MMA K step
+  static constexpr int KS = DP / 16;
+  static constexpr int LDK = DP + 8;              // row pitch of K and of a Q / O slab (halfs): conflict-free
+  static constexpr int LDV = NKP * 16 + 8;        // row pitch of V^T (halfs)
+  static constexpr int MT = (D <= 64 && NKP <= 5) ? 2 : 1;  // 16-row tiles per warp (register budget)
+  static constexpr int WROWS = 16 * MT;
+  static constexpr int ROWS = AT_WARPS * WROWS;   // query rows per CTA
+  static constexpr int NT = 2 * NKP;              // 8-key tiles
+  static constexpr int SM_K = NKP * 16 * LDK * 2;
+  static constexpr int SM_Q = AT_WARPS * WROWS * LDK * 2;
+  static constexpr int SM_V = D * LDV * 2 + D * 4;
+  static constexpr int SMEM1 = SM_K + SM_Q;
+  static constexpr int SMEM2 = SM_K + SM_Q + SM_V;
+};
 
 struct AttnArgs {
   const __half* Q;
@@ -54,115 +75,137 @@ __device__ __forceinline__ int scope_index(const AttnArgs& a, int b, int h) {
   return a.gran == DGQ_SCALE_PER_PROMPT ? b : (a.gran == DGQ_SCALE_PER_PROMPT_HEAD ? b * a.H + h : 0);
 }
 
-// Base-2 logits of 16 query rows against all keys: S[nt][0..1] = row lane/4, keys 8 nt + 2 (lane%4) + {0,1};
-// S[nt][2..3] = row lane/4 + 8.  Keys >= nk get -inf.
+// K of one head into shared memory, rows and features beyond the real ones zero.
 template <int D, int NKP>
-__device__ __forceinline__ void logits_16rows(const AttnArgs& a, const __half* q_base, int64_t q_stride,
-                                              int rows_valid, const __half* sK, float (&S)[2 * NKP][4]) {
-  constexpr int DP = (D + 15) / 16 * 16;
-  constexpr int KS = DP / 16;
-  constexpr int LDK = DP + 8;  // padded row length of K in shared memory (halfs): conflict-free fragment reads
+__device__ __forceinline__ void stage_k(const AttnArgs& a, int b, int h, __half* sK) {
+  using Cfg = AttnCfg<D, NKP>;
+  constexpr int VEC = Cfg::LDK / 8;  // 16-byte pieces per row, padding included
+  for (int i = threadIdx.x; i < NKP * 16 * VEC; i += AT_THREADS) {
+    const int j = i / VEC, v = i - j * VEC;
+    uint4 x = make_uint4(0, 0, 0, 0);
+    if (j < a.nk && v < D / 8)
+      x = __ldg(reinterpret_cast<const uint4*>(a.K + (((int64_t)b * a.nk + j) * a.H + h) * D) + v);
+    *reinterpret_cast<uint4*>(sK + j * Cfg::LDK + v * 8) = x;
+  }
+}
+
+// The warp's query rows into its slab, rows beyond the valid ones and features beyond D zero.
+template <int D, int NKP>
+__device__ __forceinline__ void stage_q(const __half* q_base, int64_t q_stride, int rows_valid, __half* slab) {
+  using Cfg = AttnCfg<D, NKP>;
+  constexpr int VEC = Cfg::DP / 8;
+  const int lane = threadIdx.x & 31;
+  for (int i = lane; i < Cfg::WROWS * VEC; i += 32) {
+    const int r = i / VEC, v = i - r * VEC;
+    uint4 x = make_uint4(0, 0, 0, 0);
+    if (r < rows_valid && v < D / 8) x = __ldg(reinterpret_cast<const uint4*>(q_base + r * q_stride) + v);
+    *reinterpret_cast<uint4*>(slab + r * Cfg::LDK + v * 8) = x;
+  }
+  __syncwarp();
+}
+
+// Base-2 logits of the warp's rows against all keys.  S[mt][nt][0..1]: row 16 mt + lane/4, keys
+// 8 nt + 2 (lane%4) + {0,1}; S[mt][nt][2..3]: row + 8.  Keys >= nk get -inf.
+template <int D, int NKP>
+__device__ __forceinline__ void logits_warp(const AttnArgs& a, const __half* slab, const __half* sK,
+                                            float (&S)[AttnCfg<D, NKP>::MT][2 * NKP][4]) {
+  using Cfg = AttnCfg<D, NKP>;
   const int lane = threadIdx.x & 31;
   const int r = lane >> 2, c = lane & 3;
 #pragma unroll
-  for (int nt = 0; nt < 2 * NKP; ++nt)
+  for (int mt = 0; mt < Cfg::MT; ++mt)
 #pragma unroll
-    for (int i = 0; i < 4; ++i) S[nt][i] = 0.f;
+    for (int nt = 0; nt < Cfg::NT; ++nt)
 #pragma unroll
-  for (int kk = 0; kk < KS; ++kk) {
-    uint32_t af[4];
+      for (int i = 0; i < 4; ++i) S[mt][nt][i] = 0.f;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int row = r + (i & 1) * 8;
-      const int col = kk * 16 + 2 * c + (i >> 1) * 8;
-      af[i] = (row < rows_valid && col < D)
-                  ? __ldg(reinterpret_cast<const uint32_t*>(q_base + row * q_stride + col))
-                  : 0u;
-    }
+  for (int kk = 0; kk < Cfg::KS; ++kk) {
+    uint32_t af[Cfg::MT][4];
 #pragma unroll
-    for (int nt = 0; nt < 2 * NKP; ++nt) {
-      const __half* kp = sK + (nt * 8 + r) * LDK + kk * 16 + 2 * c;
+    for (int mt = 0; mt < Cfg::MT; ++mt)
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        af[mt][i] = *reinterpret_cast<const uint32_t*>(slab + (mt * 16 + r + (i & 1) * 8) * Cfg::LDK + kk * 16 +
+                                                       2 * c + (i >> 1) * 8);
+#pragma unroll
+    for (int nt = 0; nt < Cfg::NT; ++nt) {
+      const __half* kp = sK + (nt * 8 + r) * Cfg::LDK + kk * 16 + 2 * c;
       const uint32_t b0 = *reinterpret_cast<const uint32_t*>(kp);
       const uint32_t b1 = *reinterpret_cast<const uint32_t*>(kp + 8);
-      mma_f16(S[nt], af[0], af[1], af[2], af[3], b0, b1);
+#pragma unroll
+      for (int mt = 0; mt < Cfg::MT; ++mt) mma_f16(S[mt][nt], af[mt][0], af[mt][1], af[mt][2], af[mt][3], b0, b1);
     }
   }
 #pragma unroll
-  for (int nt = 0; nt < 2 * NKP; ++nt)
+  for (int mt = 0; mt < Cfg::MT; ++mt)
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int key = nt * 8 + 2 * c + (i & 1);
-      S[nt][i] = key < a.nk ? S[nt][i] * a.qk_scale_log2 : -INFINITY;
-    }
+    for (int nt = 0; nt < Cfg::NT; ++nt)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int key = nt * 8 + 2 * c + (i & 1);
+        S[mt][nt][i] = key < a.nk ? S[mt][nt][i] * a.qk_scale_log2 : -INFINITY;
+      }
 }
 
 template <int D, int NKP>
-__device__ __forceinline__ void stage_k(const AttnArgs& a, int b, int h, __half* sK) {
-  constexpr int DP = (D + 15) / 16 * 16;
-  constexpr int LDK = DP + 8;
-  // zero everything (padding keys and features), then copy the head's keys with 128-bit loads
-  for (int i = threadIdx.x; i < NKP * 16 * LDK / 8; i += AT_THREADS) reinterpret_cast<uint4*>(sK)[i] = make_uint4(0, 0, 0, 0);
-  __syncthreads();
-  const int vec = D / 8;
-  for (int i = threadIdx.x; i < a.nk * vec; i += AT_THREADS) {
-    const int j = i / vec, v = i - j * vec;
-    const uint4 x = __ldg(reinterpret_cast<const uint4*>(a.K + (((int64_t)b * a.nk + j) * a.H + h) * D) + v);
-    *reinterpret_cast<uint4*>(sK + j * LDK + v * 8) = x;
-  }
-}
-
-template <int D, int NKP>
-__global__ void __launch_bounds__(AT_THREADS) attn_phase1_kernel(const AttnArgs a) {
-  constexpr int DP = (D + 15) / 16 * 16;
-  constexpr int LDK = DP + 8;
+__global__ void __launch_bounds__(AT_THREADS, 2) attn_phase1_kernel(const AttnArgs a) {
+  using Cfg = AttnCfg<D, NKP>;
   extern __shared__ __align__(16) unsigned char at_smem[];
-  __half* sK = reinterpret_cast<__half*>(at_smem);  // [NKP * 16][LDK]
+  __half* sK = reinterpret_cast<__half*>(at_smem);
+  __half* sQ = reinterpret_cast<__half*>(at_smem + Cfg::SM_K);
   const int blk = blockIdx.x;
   const int rb = blk % a.n_row_blocks;
   const int h = (blk / a.n_row_blocks) % a.H;
   const int b = blk / (a.n_row_blocks * a.H);
-  stage_k<D, NKP>(a, b, h, sK);
-  __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = lane >> 2, c = lane & 3;
-  const int row0 = rb * AT_ROWS + warp * 16;
-  const int rows_valid = min(16, a.nq - row0);
+  const int row0 = rb * Cfg::ROWS + warp * Cfg::WROWS;
+  const int rows_valid = min(Cfg::WROWS, a.nq - row0);
+  const int64_t q_stride = (int64_t)a.H * D;
+  __half* slab = sQ + warp * Cfg::WROWS * Cfg::LDK;
+  stage_k<D, NKP>(a, b, h, sK);
+  if (rows_valid > 0) stage_q<D, NKP>(a.Q + (((int64_t)b * a.nq + row0) * a.H + h) * D, q_stride, rows_valid, slab);
+  __syncthreads();
   float best = -INFINITY;
   if (rows_valid > 0) {
-    const int64_t q_stride = (int64_t)a.H * D;
-    const __half* q_base = a.Q + (((int64_t)b * a.nq + row0) * a.H + h) * D;
-    float S[2 * NKP][4];
-    logits_16rows<D, NKP>(a, q_base, q_stride, rows_valid, sK, S);
+    float S[Cfg::MT][Cfg::NT][4];
+    logits_warp<D, NKP>(a, slab, sK, S);
 #pragma unroll
-    for (int hi = 0; hi < 2; ++hi) {  // hi = 0: row r, hi = 1: row r + 8
-      float tmax = -INFINITY, trest = -INFINITY;
+    for (int mt = 0; mt < Cfg::MT; ++mt)
 #pragma unroll
-      for (int nt = 0; nt < 2 * NKP; ++nt)
+      for (int hi = 0; hi < 2; ++hi) {  // hi = 0: row r, hi = 1: row r + 8
+        float tmax = -INFINITY, trest = -INFINITY;
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          const float t = S[nt][hi * 2 + i];
-          tmax = fmaxf(tmax, t);
-          const bool is_start = (nt == 0) && (c == 0) && (i == 0);
-          if (!is_start) trest = fmaxf(trest, t);
+        for (int nt = 0; nt < Cfg::NT; ++nt)
+#pragma unroll
+          for (int i = 0; i < 2; ++i) {
+            const float t = S[mt][nt][hi * 2 + i];
+            if (nt == 0 && i == 0) {
+              tmax = fmaxf(tmax, t);
+              if (c != 0) trest = fmaxf(trest, t);  // key 0 (lane c == 0) is the <start> column
+            } else {
+              trest = fmaxf(trest, t);
+            }
+          }
+        tmax = fmaxf(tmax, trest);
+        tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+        tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+        trest = fmaxf(trest, __shfl_xor_sync(0xffffffffu, trest, 1));
+        trest = fmaxf(trest, __shfl_xor_sync(0xffffffffu, trest, 2));
+        float z = 0.f;
+#pragma unroll
+        for (int nt = 0; nt < Cfg::NT; ++nt)
+#pragma unroll
+          for (int i = 0; i < 2; ++i) z += ex2_approx(S[mt][nt][hi * 2 + i] - tmax);
+        z += __shfl_xor_sync(0xffffffffu, z, 1);
+        z += __shfl_xor_sync(0xffffffffu, z, 2);
+        const float lz = log2f(z);
+        const int row = mt * 16 + r + hi * 8;
+        if (row < rows_valid) {
+          if (c == 0) a.stats[((int64_t)b * a.H + h) * a.nq + row0 + row] = make_float2(tmax, lz);
+          best = fmaxf(best, (trest - tmax) - lz);  // log2 of the row's largest off-<start> score
         }
-      tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
-      tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
-      trest = fmaxf(trest, __shfl_xor_sync(0xffffffffu, trest, 1));
-      trest = fmaxf(trest, __shfl_xor_sync(0xffffffffu, trest, 2));
-      float z = 0.f;
-#pragma unroll
-      for (int nt = 0; nt < 2 * NKP; ++nt)
-#pragma unroll
-        for (int i = 0; i < 2; ++i) z += ex2_approx(S[nt][hi * 2 + i] - tmax);
-      z += __shfl_xor_sync(0xffffffffu, z, 1);
-      z += __shfl_xor_sync(0xffffffffu, z, 2);
-      const float lz = log2f(z);
-      const int row = r + hi * 8;
-      if (row < rows_valid) {
-        if (c == 0) a.stats[((int64_t)b * a.H + h) * a.nq + row0 + row] = make_float2(tmax, lz);
-        best = fmaxf(best, (trest - tmax) - lz);  // log2 of the row's largest off-<start> score
       }
-    }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, o));
@@ -170,31 +213,45 @@ __global__ void __launch_bounds__(AT_THREADS) attn_phase1_kernel(const AttnArgs 
     atomicMax(&a.smax[scope_index(a, b, h)], float_to_ordered(best));
 }
 
-template <int D, int NKP>
-__global__ void __launch_bounds__(AT_THREADS) attn_phase2_kernel(const AttnArgs a) {
-  constexpr int DP = (D + 15) / 16 * 16;
-  constexpr int LDK = DP + 8;
-  constexpr int LDV = NKP * 16 + 8;  // padded row length of V^T in shared memory (halfs)
+template <int D, int NKP, bool CODES>
+__global__ void __launch_bounds__(AT_THREADS, 2) attn_phase2_kernel(const AttnArgs a) {
+  using Cfg = AttnCfg<D, NKP>;
   constexpr int NT_O = D / 8;
   extern __shared__ __align__(16) unsigned char at_smem[];
-  __half* sK = reinterpret_cast<__half*>(at_smem);  // [NKP * 16][LDK]
-  __half* sVt = sK + NKP * 16 * LDK;                // [D][LDV]
+  __half* sK = reinterpret_cast<__half*>(at_smem);
+  __half* sQ = reinterpret_cast<__half*>(at_smem + Cfg::SM_K);
+  __half* sVt = reinterpret_cast<__half*>(at_smem + Cfg::SM_K + Cfg::SM_Q);  // [D][LDV], column 0 zero
+  float* sV0 = reinterpret_cast<float*>(sVt + D * Cfg::LDV);                 // [D] the <start> value row
   const int blk = blockIdx.x;
   const int rb = blk % a.n_row_blocks;
   const int h = (blk / a.n_row_blocks) % a.H;
   const int b = blk / (a.n_row_blocks * a.H);
-  stage_k<D, NKP>(a, b, h, sK);
-  for (int i = threadIdx.x; i < D * LDV / 8; i += AT_THREADS) reinterpret_cast<uint4*>(sVt)[i] = make_uint4(0, 0, 0, 0);
-  __syncthreads();
-  for (int i = threadIdx.x; i < a.nk * D; i += AT_THREADS) {
-    const int j = i / D, f = i - j * D;
-    sVt[f * LDV + j] = a.V[(((int64_t)b * a.nk + j) * a.H + h) * D + f];
-  }
-  __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = lane >> 2, c = lane & 3;
-  const int row0 = rb * AT_ROWS + warp * 16;
-  const int rows_valid = min(16, a.nq - row0);
+  const int row0 = rb * Cfg::ROWS + warp * Cfg::WROWS;
+  const int rows_valid = min(Cfg::WROWS, a.nq - row0);
+  const int64_t q_stride = (int64_t)a.H * D;
+  __half* slab = sQ + warp * Cfg::WROWS * Cfg::LDK;
+  stage_k<D, NKP>(a, b, h, sK);
+  // V^T: 128-bit loads of 8 features of one key, written transposed; keys >= nk and key 0 are zero
+  for (int i = threadIdx.x; i < NKP * 16 * (D / 8); i += AT_THREADS) {
+    const int j = i / (D / 8), v = i - j * (D / 8);
+    uint4 x = make_uint4(0, 0, 0, 0);
+    if (j < a.nk) x = __ldg(reinterpret_cast<const uint4*>(a.V + (((int64_t)b * a.nk + j) * a.H + h) * D) + v);
+    const __half* xh = reinterpret_cast<const __half*>(&x);
+    if (j == 0) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        sV0[v * 8 + e] = __half2float(xh[e]);
+        sVt[(v * 8 + e) * Cfg::LDV] = __float2half(0.f);
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) sVt[(v * 8 + e) * Cfg::LDV + j] = xh[e];
+    }
+  }
+  if (rows_valid > 0) stage_q<D, NKP>(a.Q + (((int64_t)b * a.nq + row0) * a.H + h) * D, q_stride, rows_valid, slab);
+  __syncthreads();
   const int scope = scope_index(a, b, h);
   float log2s;
   if (a.fixed_scale)
@@ -205,92 +262,110 @@ __global__ void __launch_bounds__(AT_THREADS) attn_phase2_kernel(const AttnArgs 
       (a.gran == DGQ_SCALE_PER_PROMPT_HEAD || (a.gran == DGQ_SCALE_PER_PROMPT && h == 0) || (b == 0 && h == 0)))
     a.scale_out[scope] = exp2f(log2s);
   if (rows_valid <= 0) return;
-  const int64_t q_stride = (int64_t)a.H * D;
-  const __half* q_base = a.Q + (((int64_t)b * a.nq + row0) * a.H + h) * D;
-  float S[2 * NKP][4];
-  logits_16rows<D, NKP>(a, q_base, q_stride, rows_valid, sK, S);
+  float S[Cfg::MT][Cfg::NT][4];
+  logits_warp<D, NKP>(a, slab, sK, S);
+  __syncwarp();  // the slab is reused for the output rows below
 
   const float Lf = (float)((1 << a.bits) - 1);
-  uint32_t pa[NKP][4];  // A fragments of A_hat / s * 2^14 for the second product
-  float a0[2];          // the <start> score of rows r and r + 8
+  const float Lcap = fminf(Lf, AT_CODE_CAP);
+  uint32_t pa[Cfg::MT][NKP][4];  // A fragments of A_hat / s * 2^14 for the second product
+  float a0[Cfg::MT][2];          // the <start> score of rows r and r + 8
 #pragma unroll
-  for (int hi = 0; hi < 2; ++hi) {
-    const int row = min(r + hi * 8, rows_valid - 1);
-    const float2 st = a.stats[((int64_t)b * a.H + h) * a.nq + row0 + row];
-    const float base = log2s + st.x + st.y;  // code = rint(base - t)
-    float start = ex2_approx(S[0][hi * 2] - st.x - st.y);  // meaningful on the lane with c == 0
-    start = __shfl_sync(0xffffffffu, start, lane & ~3);
-    a0[hi] = start;
+  for (int mt = 0; mt < Cfg::MT; ++mt)
 #pragma unroll
-    for (int nt = 0; nt < 2 * NKP; ++nt) {
-      uint32_t packed = 0;
+    for (int hi = 0; hi < 2; ++hi) {
+      const int row = min(mt * 16 + r + hi * 8, rows_valid - 1);
+      const float2 st = __ldg(a.stats + ((int64_t)b * a.H + h) * a.nq + row0 + row);
+      const float base = log2s + st.x + st.y;  // code = rint(base - t)
+      float start = ex2_approx(S[mt][0][hi * 2] - st.x - st.y);  // meaningful on the lane with c == 0
+      a0[mt][hi] = __shfl_sync(0xffffffffu, start, lane & ~3);
 #pragma unroll
-      for (int i = 0; i < 2; ++i) {
-        const float t = S[nt][hi * 2 + i];
-        const int key = nt * 8 + 2 * c + i;
-        // -inf logits (padding keys) give +inf -> the last code; they are dropped below
-        const float code_f = fminf(fmaxf(rintf(base - t), 0.f), Lf);
-        const int code = (int)code_f;
-        uint32_t bits16 = 0;
-        if (key >= 1 && key < a.nk) {
-          const int e = (int)AT_P_SHIFT - code;  // exponent of 2^(14 - code)
-          bits16 = e >= -14 ? (uint32_t)(e + 15) << 10 : (e >= -24 ? 1u << (e + 24) : 0u);
-          if (a.codes_out && (r + hi * 8) < rows_valid)
-            a.codes_out[(((int64_t)b * a.H + h) * a.nq + row0 + r + hi * 8) * (a.nk - 1) + key - 1] = (uint8_t)code;
+      for (int nt = 0; nt < Cfg::NT; ++nt) {
+        float p[2];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const float t = S[mt][nt][hi * 2 + i];
+          // rint by adding 1.5 * 2^23: the low bits of the sum are the integer.  -inf logits (padding
+          // keys) clamp to the cap; their V^T columns are zero, as is the <start> column.
+          const float x = fminf(fmaxf(base - t, 0.f), CODES ? Lf : Lcap);
+          const int code = __float_as_int(x + 12582912.0f) - 0x4B400000;
+          if (CODES) {
+            const int key = nt * 8 + 2 * c + i;
+            const int orow = mt * 16 + r + hi * 8;
+            if (key >= 1 && key < a.nk && orow < rows_valid)
+              a.codes_out[(((int64_t)b * a.H + h) * a.nq + row0 + orow) * (a.nk - 1) + key - 1] = (uint8_t)code;
+          }
+          // 2^(14 - code) as an fp32 exponent field; beyond the cap it converts to an fp16 zero
+          p[i] = __int_as_float((127 + (int)AT_P_SHIFT - min(code, (int)AT_CODE_CAP)) << 23);
         }
-        packed |= bits16 << (16 * i);
+        const __half2 ph = __floats2half2_rn(p[0], p[1]);
+        pa[mt][nt >> 1][(nt & 1) * 2 + hi] = *reinterpret_cast<const uint32_t*>(&ph);
       }
-      pa[nt >> 1][(nt & 1) * 2 + hi] = packed;
     }
-  }
-  float acc[NT_O][4];
+  float acc[Cfg::MT][NT_O][4];
 #pragma unroll
-  for (int nt = 0; nt < NT_O; ++nt)
+  for (int mt = 0; mt < Cfg::MT; ++mt)
 #pragma unroll
-    for (int i = 0; i < 4; ++i) acc[nt][i] = 0.f;
+    for (int nt = 0; nt < NT_O; ++nt)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) acc[mt][nt][i] = 0.f;
 #pragma unroll
   for (int kk = 0; kk < NKP; ++kk)
 #pragma unroll
     for (int nt = 0; nt < NT_O; ++nt) {
-      const __half* vp = sVt + (nt * 8 + r) * LDV + kk * 16 + 2 * c;
+      const __half* vp = sVt + (nt * 8 + r) * Cfg::LDV + kk * 16 + 2 * c;
       const uint32_t b0 = *reinterpret_cast<const uint32_t*>(vp);
       const uint32_t b1 = *reinterpret_cast<const uint32_t*>(vp + 8);
-      mma_f16(acc[nt], pa[kk][0], pa[kk][1], pa[kk][2], pa[kk][3], b0, b1);
+#pragma unroll
+      for (int mt = 0; mt < Cfg::MT; ++mt)
+        mma_f16(acc[mt][nt], pa[mt][kk][0], pa[mt][kk][1], pa[mt][kk][2], pa[mt][kk][3], b0, b1);
     }
+  // O = A_i0 V_0 + s 2^-14 acc, staged in the warp's slab and written with 128-bit stores
   const float s_out = exp2f(log2s - AT_P_SHIFT);
-  __half* o_base = a.O + (((int64_t)b * a.nq + row0) * a.H + h) * D;
 #pragma unroll
   for (int nt = 0; nt < NT_O; ++nt) {
     const int col = nt * 8 + 2 * c;
-    const float v0x = __half2float(sVt[col * LDV]), v0y = __half2float(sVt[(col + 1) * LDV]);
+    const float2 v0 = *reinterpret_cast<const float2*>(sV0 + col);
 #pragma unroll
-    for (int hi = 0; hi < 2; ++hi) {
-      const int row = r + hi * 8;
-      if (row < rows_valid) {
-        const float ox = fmaf(a0[hi], v0x, s_out * acc[nt][hi * 2]);
-        const float oy = fmaf(a0[hi], v0y, s_out * acc[nt][hi * 2 + 1]);
-        *reinterpret_cast<__half2*>(o_base + row * q_stride + col) = __floats2half2_rn(ox, oy);
+    for (int mt = 0; mt < Cfg::MT; ++mt)
+#pragma unroll
+      for (int hi = 0; hi < 2; ++hi) {
+        const float ox = fmaf(a0[mt][hi], v0.x, s_out * acc[mt][nt][hi * 2]);
+        const float oy = fmaf(a0[mt][hi], v0.y, s_out * acc[mt][nt][hi * 2 + 1]);
+        *reinterpret_cast<__half2*>(slab + (mt * 16 + r + hi * 8) * Cfg::LDK + col) = __floats2half2_rn(ox, oy);
       }
-    }
+  }
+  __syncwarp();
+  __half* o_base = a.O + (((int64_t)b * a.nq + row0) * a.H + h) * D;
+  for (int i = lane; i < Cfg::WROWS * (D / 8); i += 32) {
+    const int rr = i / (D / 8), v = i - rr * (D / 8);
+    if (rr < rows_valid)
+      *(reinterpret_cast<uint4*>(o_base + rr * q_stride) + v) = *reinterpret_cast<const uint4*>(slab + rr * Cfg::LDK + v * 8);
   }
 }
 
 template <int D, int NKP>
 static dgq_status launch_attn(const AttnArgs& a, cudaStream_t stream) {
-  constexpr int DP = (D + 15) / 16 * 16;
-  constexpr int SM1 = NKP * 16 * (DP + 8) * 2;
-  constexpr int SM2 = SM1 + D * (NKP * 16 + 8) * 2;
+  using Cfg = AttnCfg<D, NKP>;
+  constexpr int SM1 = Cfg::SMEM1;
+  constexpr int SM2 = Cfg::SMEM2;
   static bool attr_set[64] = {false};
   int dev = 0;
   DGQ_CUDA_OK(cudaGetDevice(&dev));
   if (dev >= 64 || !attr_set[dev]) {
     DGQ_CUDA_OK(cudaFuncSetAttribute(attn_phase1_kernel<D, NKP>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM1));
-    DGQ_CUDA_OK(cudaFuncSetAttribute(attn_phase2_kernel<D, NKP>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM2));
+    DGQ_CUDA_OK(cudaFuncSetAttribute(attn_phase2_kernel<D, NKP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM2));
+    DGQ_CUDA_OK(cudaFuncSetAttribute(attn_phase2_kernel<D, NKP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM2));
     if (dev < 64) attr_set[dev] = true;
   }
-  const int grid = a.B * a.H * a.n_row_blocks;
-  attn_phase1_kernel<D, NKP><<<grid, AT_THREADS, SM1, stream>>>(a);
-  attn_phase2_kernel<D, NKP><<<grid, AT_THREADS, SM2, stream>>>(a);
+  AttnArgs aa = a;
+  aa.n_row_blocks = (a.nq + Cfg::ROWS - 1) / Cfg::ROWS;
+  const int grid = a.B * a.H * aa.n_row_blocks;
+  attn_phase1_kernel<D, NKP><<<grid, AT_THREADS, SM1, stream>>>(aa);
+  if (a.codes_out)
+    attn_phase2_kernel<D, NKP, true><<<grid, AT_THREADS, SM2, stream>>>(aa);
+  else
+    attn_phase2_kernel<D, NKP, false><<<grid, AT_THREADS, SM2, stream>>>(aa);
   g_launches += 2;
   DGQ_CUDA_OK(cudaGetLastError());
   return DGQ_OK;
@@ -345,7 +420,7 @@ extern "C" dgq_status dgq_cross_attn_logq(const void* Q, const void* K, const vo
   a.fixed_scale = fixed_scale;
   a.scale_out = scale_out;
   a.codes_out = codes_out;
-  a.n_row_blocks = (nq + AT_ROWS - 1) / AT_ROWS;
+  a.n_row_blocks = 0;  // set per kernel configuration at launch
   cudaStream_t st = (cudaStream_t)stream;
   // 0x80 bytes decode to about -3.4e38 in the ordered-integer encoding: "no score seen yet"
   DGQ_CUDA_OK(cudaMemsetAsync(a.smax, 0x80, attn_smax_bytes(B, H), st));
