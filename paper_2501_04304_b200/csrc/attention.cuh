@@ -75,17 +75,34 @@ __device__ __forceinline__ int scope_index(const AttnArgs& a, int b, int h) {
   return a.gran == DGQ_SCALE_PER_PROMPT ? b : (a.gran == DGQ_SCALE_PER_PROMPT_HEAD ? b * a.H + h : 0);
 }
 
-// K of one head into shared memory, rows and features beyond the real ones zero.
+// K of one head into shared memory, rows and features beyond the real ones zero.  The loads are
+// issued first (into registers) and stored later, so that other loads can be put in between and
+// all their latencies overlap.
 template <int D, int NKP>
-__device__ __forceinline__ void stage_k(const AttnArgs& a, int b, int h, __half* sK) {
-  using Cfg = AttnCfg<D, NKP>;
-  constexpr int VEC = Cfg::LDK / 8;  // 16-byte pieces per row, padding included
-  for (int i = threadIdx.x; i < NKP * 16 * VEC; i += AT_THREADS) {
+struct KStage {
+  static constexpr int VEC = AttnCfg<D, NKP>::LDK / 8;  // 16-byte pieces per row, padding included
+  static constexpr int N = (NKP * 16 * VEC + AT_THREADS - 1) / AT_THREADS;
+};
+template <int D, int NKP>
+__device__ __forceinline__ void load_k(const AttnArgs& a, int b, int h, uint4 (&x)[KStage<D, NKP>::N]) {
+  constexpr int VEC = KStage<D, NKP>::VEC;
+#pragma unroll
+  for (int e = 0; e < KStage<D, NKP>::N; ++e) {
+    const int i = threadIdx.x + e * AT_THREADS;
     const int j = i / VEC, v = i - j * VEC;
-    uint4 x = make_uint4(0, 0, 0, 0);
+    x[e] = make_uint4(0, 0, 0, 0);
     if (j < a.nk && v < D / 8)
-      x = __ldg(reinterpret_cast<const uint4*>(a.K + (((int64_t)b * a.nk + j) * a.H + h) * D) + v);
-    *reinterpret_cast<uint4*>(sK + j * Cfg::LDK + v * 8) = x;
+      x[e] = __ldg(reinterpret_cast<const uint4*>(a.K + (((int64_t)b * a.nk + j) * a.H + h) * D) + v);
+  }
+}
+template <int D, int NKP>
+__device__ __forceinline__ void store_k(const uint4 (&x)[KStage<D, NKP>::N], __half* sK) {
+  constexpr int VEC = KStage<D, NKP>::VEC;
+#pragma unroll
+  for (int e = 0; e < KStage<D, NKP>::N; ++e) {
+    const int i = threadIdx.x + e * AT_THREADS;
+    const int j = i / VEC, v = i - j * VEC;
+    if (i < NKP * 16 * VEC) *reinterpret_cast<uint4*>(sK + j * AttnCfg<D, NKP>::LDK + v * 8) = x[e];
   }
 }
 
@@ -94,12 +111,22 @@ template <int D, int NKP>
 __device__ __forceinline__ void stage_q(const __half* q_base, int64_t q_stride, int rows_valid, __half* slab) {
   using Cfg = AttnCfg<D, NKP>;
   constexpr int VEC = Cfg::DP / 8;
+  constexpr int N = (Cfg::WROWS * VEC + 31) / 32;
   const int lane = threadIdx.x & 31;
-  for (int i = lane; i < Cfg::WROWS * VEC; i += 32) {
+  uint4 x[N];  // all loads in flight before the first store
+#pragma unroll
+  for (int e = 0; e < N; ++e) {
+    const int i = lane + e * 32;
     const int r = i / VEC, v = i - r * VEC;
-    uint4 x = make_uint4(0, 0, 0, 0);
-    if (r < rows_valid && v < D / 8) x = __ldg(reinterpret_cast<const uint4*>(q_base + r * q_stride) + v);
-    *reinterpret_cast<uint4*>(slab + r * Cfg::LDK + v * 8) = x;
+    x[e] = make_uint4(0, 0, 0, 0);
+    if (i < Cfg::WROWS * VEC && r < rows_valid && v < D / 8)
+      x[e] = __ldg(reinterpret_cast<const uint4*>(q_base + r * q_stride) + v);
+  }
+#pragma unroll
+  for (int e = 0; e < N; ++e) {
+    const int i = lane + e * 32;
+    const int r = i / VEC, v = i - r * VEC;
+    if (i < Cfg::WROWS * VEC) *reinterpret_cast<uint4*>(slab + r * Cfg::LDK + v * 8) = x[e];
   }
   __syncwarp();
 }
@@ -163,8 +190,10 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_phase1_kernel(const AttnAr
   const int rows_valid = min(Cfg::WROWS, a.nq - row0);
   const int64_t q_stride = (int64_t)a.H * D;
   __half* slab = sQ + warp * Cfg::WROWS * Cfg::LDK;
-  stage_k<D, NKP>(a, b, h, sK);
+  uint4 xk[KStage<D, NKP>::N];
+  load_k<D, NKP>(a, b, h, xk);
   if (rows_valid > 0) stage_q<D, NKP>(a.Q + (((int64_t)b * a.nq + row0) * a.H + h) * D, q_stride, rows_valid, slab);
+  store_k<D, NKP>(xk, sK);
   __syncthreads();
   float best = -INFINITY;
   if (rows_valid > 0) {
@@ -232,13 +261,27 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_phase2_kernel(const AttnAr
   const int rows_valid = min(Cfg::WROWS, a.nq - row0);
   const int64_t q_stride = (int64_t)a.H * D;
   __half* slab = sQ + warp * Cfg::WROWS * Cfg::LDK;
-  stage_k<D, NKP>(a, b, h, sK);
-  // V^T: 128-bit loads of 8 features of one key, written transposed; keys >= nk and key 0 are zero
-  for (int i = threadIdx.x; i < NKP * 16 * (D / 8); i += AT_THREADS) {
+  uint4 xk[KStage<D, NKP>::N];
+  load_k<D, NKP>(a, b, h, xk);
+  // V^T: 128-bit loads of 8 features of one key, written transposed; keys >= nk and key 0 are zero.
+  // K, V and Q are all requested before anything is written, so their latencies overlap.
+  constexpr int NV = (NKP * 16 * (D / 8) + AT_THREADS - 1) / AT_THREADS;
+  uint4 xv[NV];
+#pragma unroll
+  for (int e = 0; e < NV; ++e) {
+    const int i = threadIdx.x + e * AT_THREADS;
     const int j = i / (D / 8), v = i - j * (D / 8);
-    uint4 x = make_uint4(0, 0, 0, 0);
-    if (j < a.nk) x = __ldg(reinterpret_cast<const uint4*>(a.V + (((int64_t)b * a.nk + j) * a.H + h) * D) + v);
-    const __half* xh = reinterpret_cast<const __half*>(&x);
+    xv[e] = make_uint4(0, 0, 0, 0);
+    if (j < a.nk) xv[e] = __ldg(reinterpret_cast<const uint4*>(a.V + (((int64_t)b * a.nk + j) * a.H + h) * D) + v);
+  }
+  if (rows_valid > 0) stage_q<D, NKP>(a.Q + (((int64_t)b * a.nq + row0) * a.H + h) * D, q_stride, rows_valid, slab);
+  store_k<D, NKP>(xk, sK);
+#pragma unroll
+  for (int ev = 0; ev < NV; ++ev) {
+    const int i = threadIdx.x + ev * AT_THREADS;
+    if (i >= NKP * 16 * (D / 8)) continue;
+    const int j = i / (D / 8), v = i - j * (D / 8);
+    const __half* xh = reinterpret_cast<const __half*>(&xv[ev]);
     if (j == 0) {
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
@@ -250,7 +293,6 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_phase2_kernel(const AttnAr
       for (int e = 0; e < 8; ++e) sVt[(v * 8 + e) * Cfg::LDV + j] = xh[e];
     }
   }
-  if (rows_valid > 0) stage_q<D, NKP>(a.Q + (((int64_t)b * a.nq + row0) * a.H + h) * D, q_stride, rows_valid, slab);
   __syncthreads();
   const int scope = scope_index(a, b, h);
   float log2s;

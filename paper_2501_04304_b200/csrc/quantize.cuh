@@ -73,10 +73,26 @@ __global__ void __launch_bounds__(QA_THREADS) quantize_act_kernel(const QuantArg
   const int64_t warps_total = (int64_t)gridDim.x * QA_WARPS;
   for (int64_t row0 = ((int64_t)blockIdx.x * QA_WARPS + warp) * rpw; row0 < a.M; row0 += warps_total * rpw) {
     const int rows = (int)min((int64_t)rpw, a.M - row0);
-    for (int r = 0; r < rows; ++r) {
-      const uint4* src = reinterpret_cast<const uint4*>(a.X + (row0 + r) * a.ld);
-      uint4* dst = reinterpret_cast<uint4*>(rows_s + r * a.C);
-      for (int v = lane; v < vec_per_row; v += 32) dst[v] = __ldg(src + v);
+    // Row loads in batches of eight 128-bit pieces per lane: every load of a batch is issued before
+    // the first store, so the memory latency is paid once per batch and not once per piece.
+    {
+      const int n_vec = rows * vec_per_row;
+      for (int v0 = 0; v0 < n_vec; v0 += 8 * 32) {
+        uint4 x[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int i = v0 + e * 32 + lane;
+          if (i < n_vec) {
+            const int r = i / vec_per_row, v = i - r * vec_per_row;
+            x[e] = __ldg(reinterpret_cast<const uint4*>(a.X + (row0 + r) * a.ld) + v);
+          }
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int i = v0 + e * 32 + lane;
+          if (i < n_vec) reinterpret_cast<uint4*>(rows_s)[i] = x[e];  // rows are packed: pitch C halfs
+        }
+      }
     }
     if (a.dynamic)
       for (int i = lane; i < rows * a.G; i += 32) {
