@@ -45,6 +45,7 @@ constexpr int GEMM_THREADS_W8 = 19 * 32;
 constexpr int GEMM_UNPACK_WARPS = 3;
 constexpr int GEMM_UNPACK_THREADS = GEMM_UNPACK_WARPS * 32;
 constexpr int GEMM_THREADS_W4 = GEMM_THREADS_W8 + GEMM_UNPACK_THREADS;
+constexpr int GEMM_MAX_ATOMS = 1024;           // 32768 reduction positions
 constexpr int GEMM_A_STAGE = GEMM_BM * 128;  // bytes
 constexpr int GEMM_SMEM_LIMIT = 227 * 1024;
 
@@ -85,6 +86,7 @@ struct GemmArgs {
   const __half* bias;         // [N] or null
   const uint8_t* w_packed;    // 4-bit weights [N_pad][Kt/2]
   int seg_end[DGQ_MAX_GROUPS];    // end atom of every group segment
+  unsigned long long end_mask[GEMM_MAX_ATOMS / 64];  // bit i: atom i is the last of its group
   // conv
   int conv_W, conv_H;
   int grp_atoms[DGQ_MAX_GROUPS];  // channel atoms of every group
@@ -165,9 +167,13 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   if (warp == GEMM_WARP_TMA) {
     // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      tma_prefetch_desc(&tmA);
-      if (!W4) tma_prefetch_desc(&tmB);
+    // The whole warp walks the loop (so that no lane of it is parked at the final CTA barrier while
+    // another one spins); lane 0 issues the copies.
+    {
+      if (lane == 0) {
+        tma_prefetch_desc(&tmA);
+        if (!W4) tma_prefetch_desc(&tmB);
+      }
       uint32_t it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
@@ -185,12 +191,12 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int ks = 0; ks < n_kstages && ok; ++ks, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
-          ok = mbar_wait(&sh->empty[s], ph ^ 1, abort_flag);
+          ok = __all_sync(0xffffffffu, mbar_wait(&sh->empty[s], ph ^ 1, abort_flag));
           if (!ok) break;
           const int atoms_here = min(4, n_atoms - ks * 4);
           uint32_t bytes = W4 ? 0u : (uint32_t)Cfg::B_STAGE;
           bytes += CONV ? (uint32_t)(atoms_here * 4096) : (uint32_t)GEMM_A_STAGE;
-          mbar_arrive_expect_tx(&sh->full[s], bytes);
+          if (lane == 0) mbar_arrive_expect_tx(&sh->full[s], bytes);
           if (CONV) {
             for (int j = 0; j < atoms_here; ++j) {
               const int atom = ks * 4 + j;
@@ -202,53 +208,79 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               const int tap = local / a.grp_atoms[g];
               const int ca = local - tap * a.grp_atoms[g];
               const int ky = tap / 3, kx = tap - ky * 3;
-              tma_load_4d(smA + s * GEMM_A_STAGE + j * 4096, &tmA, &sh->full[s], a.grp_chan0[g] + ca * 32,
-                          cw + kx - 1, chh + ky - 1, cn);
+              if (lane == 0)
+                tma_load_4d(smA + s * GEMM_A_STAGE + j * 4096, &tmA, &sh->full[s], a.grp_chan0[g] + ca * 32,
+                            cw + kx - 1, chh + ky - 1, cn);
             }
           } else {
-            tma_load_2d(smA + s * GEMM_A_STAGE, &tmA, &sh->full[s], ks * 128, m0);
+            if (lane == 0) tma_load_2d(smA + s * GEMM_A_STAGE, &tmA, &sh->full[s], ks * 128, m0);
           }
-          if (!W4) tma_load_2d(smB + s * Cfg::B_STAGE, &tmB, &sh->full[s], ks * 128, n0);
+          if (!W4 && lane == 0) tma_load_2d(smB + s * Cfg::B_STAGE, &tmB, &sh->full[s], ks * 128, n0);
+          __syncwarp();
         }
       }
     }
   } else if (warp == GEMM_WARP_MMA) {
     // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      uint32_t it = 0, acc_it = 0;
+    {
+      // The issuing thread is a single lane: its dependent instruction chain per MMA is what bounds
+      // short groups, so everything that can be is precomputed (descriptor words, the per-stage
+      // bit mask of atoms that end a group, running accumulator index and parity).
+      constexpr uint32_t A_HI = CONV ? smem_desc_hi(256, 6) : smem_desc_hi(1024, 2);
+      constexpr uint32_t B_HI = smem_desc_hi(1024, 2);
+      const uint32_t a_lo0 = smem_desc_lo(smem_u32(smA)), b_lo0 = smem_desc_lo(smem_u32(smB));
+      const uint32_t idesc = a.idesc;
+      uint32_t it = 0;
+      int s = 0;                 // stage slot of `it`
+      uint32_t full_phase = 0;   // parity of the slot's next "full" phase
+      int ab = 0;                // accumulator of the next group
+      uint32_t acc_phase = 1;    // parity to wait for on its "empty" barrier (fresh barriers pass)
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-        int g = 0;
         bool need_acc = true;  // the next atom starts a group: take the next accumulator first
-        int ab = 0;
+        uint32_t d_tmem = tmem_base;
+        uint64_t ends = 0;     // bit i: atom (16 * 4) * word + i is the last of its group
         for (int ks = 0; ks < n_kstages && ok; ++ks, ++it) {
-          const int s = it % STAGES;
-          ok = mbar_wait(&sh->full[s], (it / STAGES) & 1, abort_flag);
+          if ((ks & 15) == 0) ends = a.end_mask[ks >> 4];
+          const uint32_t end_bits = (uint32_t)(ends >> ((ks & 15) * 4)) & 0xFu;
+          ok = __all_sync(0xffffffffu, mbar_wait(&sh->full[s], full_phase, abort_flag));
           if (!ok) break;
           tc_fence_after();
           const int atoms_here = min(4, n_atoms - ks * 4);
-          const uint32_t a_addr = smem_u32(smA + s * GEMM_A_STAGE);
-          const uint32_t b_addr = smem_u32(smB + s * Cfg::B_STAGE);
-          for (int j = 0; j < atoms_here && ok; ++j) {
-            const int atom = ks * 4 + j;
-            if (need_acc) {
-              ab = acc_it % NACC;
-              ok = mbar_wait(&sh->acc_empty[ab], ((acc_it / NACC) & 1) ^ 1, abort_flag);
-              if (!ok) break;
-              tc_fence_after();
-            }
-            const uint64_t da = CONV ? smem_desc(a_addr + j * 4096, 256, 6) : smem_desc(a_addr + j * 32, 1024, 2);
-            const uint64_t db = smem_desc(b_addr + j * 32, 1024, 2);
-            mma_i8(tmem_base + (uint32_t)(ab * BN), da, db, a.idesc, need_acc ? 0u : 1u);
-            need_acc = false;
-            if (atom + 1 == a.seg_end[g]) {  // last atom of the group: hand the accumulator over right away
-              mma_commit(&sh->acc_full[ab]);
-              ++acc_it;
-              ++g;
-              need_acc = true;
+          const uint32_t a_lo = a_lo0 + (uint32_t)s * (GEMM_A_STAGE >> 4);
+          const uint32_t b_lo = b_lo0 + (uint32_t)s * (Cfg::B_STAGE >> 4);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            if (j < atoms_here && ok) {
+              if (need_acc) {
+                ok = __all_sync(0xffffffffu, mbar_wait(&sh->acc_empty[ab], acc_phase, abort_flag));
+                if (ok) {
+                  tc_fence_after();
+                  d_tmem = tmem_base + (uint32_t)(ab * BN);
+                }
+              }
+              if (ok) {
+                if (lane == 0)
+                  mma_i8_lohi(d_tmem, a_lo + (CONV ? j * 256 : j * 2), A_HI, b_lo + j * 2, B_HI, idesc,
+                              need_acc ? 0u : 1u);
+                need_acc = false;
+                if (end_bits & (1u << j)) {  // last atom of the group: hand the accumulator over right away
+                  if (lane == 0) mma_commit(&sh->acc_full[ab]);
+                  if (++ab == NACC) {
+                    ab = 0;
+                    acc_phase ^= 1u;
+                  }
+                  need_acc = true;
+                }
+              }
             }
           }
-          if (ok) mma_commit(&sh->empty[s]);  // stage reusable once these MMAs have read it
+          if (ok && lane == 0) mma_commit(&sh->empty[s]);  // stage reusable once these MMAs have read it
+          __syncwarp();
+          if (++s == STAGES) {
+            s = 0;
+            full_phase ^= 1u;
+          }
         }
       }
     }
@@ -330,10 +362,9 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (a.use_zp) {
           // rare: Z outside the code range (the stored padding code is the clamped Z), or a group
           // whose padding could not absorb all of wsum
-          const int Zc = min(max(Z, 0), a.code_max);
-          const float c1 = -s * (float)(Z - Zc);
-          const float c2 = ((a.res_mask >> g) & 1u) ? -s * (float)Zc : 0.f;
-          if (__any_sync(0xffffffffu, c1 != 0.f)) {
+          if (__any_sync(0xffffffffu, (uint32_t)Z > (uint32_t)a.code_max)) {
+            const int Zc = min(max(Z, 0), a.code_max);
+            const float c1 = -s * (float)(Z - Zc);
             const float4* ws = reinterpret_cast<const float4*>(wsum_s + g * BN + sl * CW);
 #pragma unroll
             for (int i = 0; i < CW; i += 4) {
@@ -345,6 +376,7 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
           }
           if ((a.res_mask >> g) & 1u) {
+            const float c2 = -s * (float)min(max(Z, 0), a.code_max);
             const float4* wr = reinterpret_cast<const float4*>(a.wres + (size_t)g * a.N_pad + col0);
 #pragma unroll
             for (int i = 0; i < CW; i += 4) {
@@ -382,23 +414,26 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   } else if (warp == GEMM_WARP_STORE) {
     // ------------------------------------------------------------ output store
-    if (lane == 0) {
-      tma_prefetch_desc(&tmY);
+    {
+      if (lane == 0) tma_prefetch_desc(&tmY);
       uint32_t tile_it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tile_it) {
         const int tm = tile / a.n_tiles_n, tn = tile - tm * a.n_tiles_n;
         const int n0 = tn * BN;
-        ok = mbar_wait(&sh->out_full, tile_it & 1, abort_flag);
+        ok = __all_sync(0xffffffffu, mbar_wait(&sh->out_full, tile_it & 1, abort_flag));
         if (!ok) break;
+        if (lane == 0) {
 #pragma unroll
-        for (int pnl = 0; pnl < BN / 32; ++pnl)
-          if (n0 + pnl * 32 < a.N) tma_store_2d(&tmY, smOut + pnl * (GEMM_BM * 64), n0 + pnl * 32, tm * GEMM_BM);
-        bulk_commit();
-        bulk_wait_read0();
-        mbar_arrive(&sh->out_free);
+          for (int pnl = 0; pnl < BN / 32; ++pnl)
+            if (n0 + pnl * 32 < a.N) tma_store_2d(&tmY, smOut + pnl * (GEMM_BM * 64), n0 + pnl * 32, tm * GEMM_BM);
+          bulk_commit();
+          bulk_wait_read0();
+          mbar_arrive(&sh->out_free);
+        }
+        __syncwarp();
       }
-      bulk_wait0();
+      if (lane == 0) bulk_wait0();
     }
   } else if (W4) {
     // ------------------------------------------------------------ 4-bit weight unpack into the B stage
@@ -584,6 +619,8 @@ extern "C" dgq_status dgq_linear(const dgq_groups* g, const dgq_weight* w, int t
   a.wsum = w->d_wsum;
   a.bias = (const __half*)bias;
   a.w_packed = (const uint8_t*)w->d_w;
+  if (w->Kt / DGQ_K_ATOM > GEMM_MAX_ATOMS) return DGQ_ERR_UNSUPPORTED;
+  for (int k = 0; k < g->G; ++k) a.end_mask[(w->seg_end[k] - 1) >> 6] |= 1ull << ((w->seg_end[k] - 1) & 63);
   for (int k = 0; k < g->G; ++k) {
     a.seg_end[k] = w->seg_end[k];
     a.grp_atoms[k] = (g->group_off[k + 1] - g->group_off[k]) / DGQ_K_ATOM;
