@@ -46,7 +46,7 @@ __device__ __forceinline__ void load_chunk_perm(const int16_t* perm, int ch, int
   }
 }
 
-__global__ void __launch_bounds__(QA_THREADS) quantize_act_kernel(const QuantArgs a) {
+__global__ void __launch_bounds__(QA_THREADS, 4) quantize_act_kernel(const QuantArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int n_chunks = a.K_pad >> 4;
   // layout: perm [K_pad] int16 | chunk_group [n_chunks] u8 | per warp: rows [rpw][C] fp16, cells [rpw][G] x 4 ints
@@ -73,14 +73,14 @@ __global__ void __launch_bounds__(QA_THREADS) quantize_act_kernel(const QuantArg
   const int64_t warps_total = (int64_t)gridDim.x * QA_WARPS;
   for (int64_t row0 = ((int64_t)blockIdx.x * QA_WARPS + warp) * rpw; row0 < a.M; row0 += warps_total * rpw) {
     const int rows = (int)min((int64_t)rpw, a.M - row0);
-    // Row loads in batches of eight 128-bit pieces per lane: every load of a batch is issued before
+    // Row loads in batches of four 128-bit pieces per lane: every load of a batch is issued before
     // the first store, so the memory latency is paid once per batch and not once per piece.
     {
       const int n_vec = rows * vec_per_row;
-      for (int v0 = 0; v0 < n_vec; v0 += 8 * 32) {
-        uint4 x[8];
+      for (int v0 = 0; v0 < n_vec; v0 += 4 * 32) {
+        uint4 x[4];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
+        for (int e = 0; e < 4; ++e) {
           const int i = v0 + e * 32 + lane;
           if (i < n_vec) {
             const int r = i / vec_per_row, v = i - r * vec_per_row;
@@ -88,7 +88,7 @@ __global__ void __launch_bounds__(QA_THREADS) quantize_act_kernel(const QuantArg
           }
         }
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
+        for (int e = 0; e < 4; ++e) {
           const int i = v0 + e * 32 + lane;
           if (i < n_vec) reinterpret_cast<uint4*>(rows_s)[i] = x[e];  // rows are packed: pitch C halfs
         }
