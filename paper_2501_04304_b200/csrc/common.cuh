@@ -109,6 +109,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
+// Same test, but the hardware may park the thread for up to `ns` nanoseconds while the phase is
+// still pending, so a waiting warp does not compete for issue slots with the working ones.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint64_t* bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
+      : "memory");
+  return ok != 0;
+}
+
 // Bounded wait: gives up after about a second (2^31 SM clocks) or as soon as another
 // thread of the CTA has raised `*abort_flag`.  Returns false when it gave up; the caller
 // must then leave through the kernel's common exit path.
@@ -117,7 +131,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   const long long t0 = clock64();
   uint32_t spins = 0;
   while (true) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait_parked(bar, parity, 4000u)) return true;
     if ((++spins & 63u) == 0) {
       if (*abort_flag) return false;
       if (clock64() - t0 > (1ll << 31)) {
@@ -127,6 +141,90 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
       }
     }
   }
+}
+
+// Bounded wait without a return value, for hot loops: after 2^21 parked polls (of at most a
+// microsecond each) it records a time-out and raises `*abort_flag`; once the flag is up every wait
+// returns at its first failed poll.  The caller tests the flag at a coarser grain (once per tile)
+// and leaves through the kernel's common exit path; what it does in between only touches memory
+// the CTA owns.
+__device__ __forceinline__ void mbar_wait_lean(uint32_t bar_addr, uint32_t parity, volatile int* abort_flag) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar_addr), "r"(parity)
+      : "memory");
+  if (ok) return;
+  if (*abort_flag) return;
+  for (uint32_t spins = 0; spins < (1u << 21); ++spins) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar_addr), "r"(parity), "r"(1000u)
+        : "memory");
+    if (ok) return;
+    if ((spins & 31u) == 31u && *abort_flag) return;
+  }
+  *abort_flag = 1;
+  record_error(DGQ_ERR_TIMEOUT);
+}
+// One non-blocking poll; the result can be consumed many instructions later.
+__device__ __forceinline__ uint32_t mbar_try_addr(uint32_t bar_addr, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar_addr), "r"(parity)
+      : "memory");
+  return ok;
+}
+// Register re-balancing between the warpgroups of a CTA (every warp of an aligned group of four
+// executes the same instruction).
+template <int REGS>
+__device__ __forceinline__ void reg_alloc() {
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS));
+}
+template <int REGS>
+__device__ __forceinline__ void reg_dealloc() {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS));
+}
+__device__ __forceinline__ void mbar_arrive_addr(uint32_t bar_addr) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_addr) : "memory");
+}
+
+// Two fp32 lanes in one 64-bit register (the operand form of the packed fp32 instructions).
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+// y += s * float(i) on two lanes: two conversions and one packed fused multiply-add.
+__device__ __forceinline__ void cvt_fma_f32x2(unsigned long long& y, unsigned long long s2, uint32_t i0, uint32_t i1) {
+  asm volatile("{\n\t.reg .f32 f0, f1;\n\t.reg .b64 t;\n\t"
+      "cvt.rn.f32.s32 f0, %1;\n\t"
+      "cvt.rn.f32.s32 f1, %2;\n\t"
+      "mov.b64 t, {f0, f1};\n\t"
+      "fma.rn.f32x2 %0, %3, t, %0;\n\t}"
+      : "+l"(y)
+      : "r"(i0), "r"(i1), "l"(s2));
+}
+
+// d = a * b + c on two lanes
+__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b,
+                                                        unsigned long long c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
 }
 
 __device__ __forceinline__ void fence_barrier_init() {
@@ -219,6 +317,10 @@ __device__ __forceinline__ constexpr uint32_t smem_desc_hi(uint32_t sbo_bytes, u
 // Arrives on `bar` once every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void mma_commit_addr(uint32_t bar_addr) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_addr)
                : "memory");
 }
 // 32 lanes x 16 consecutive 32-bit columns: thread i of the warp receives row (lane base + i).

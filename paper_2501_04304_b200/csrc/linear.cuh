@@ -36,15 +36,24 @@
 namespace dgq {
 
 constexpr int GEMM_BM = 128;
-constexpr int GEMM_EPI_WARPS = 16;
-constexpr int GEMM_EPI_THREADS = GEMM_EPI_WARPS * 32;
-constexpr int GEMM_WARP_TMA = 16;
-constexpr int GEMM_WARP_MMA = 17;
-constexpr int GEMM_WARP_STORE = 18;
-constexpr int GEMM_THREADS_W8 = 19 * 32;
-constexpr int GEMM_UNPACK_WARPS = 3;
+constexpr int GEMM_UNPACK_WARPS = 5;
 constexpr int GEMM_UNPACK_THREADS = GEMM_UNPACK_WARPS * 32;
-constexpr int GEMM_THREADS_W4 = GEMM_THREADS_W8 + GEMM_UNPACK_THREADS;
+// Eight epilogue warps (two aligned groups of four: a warp reads the TMEM lane quarter warp % 4),
+// then the producer, issuer and store warps and, for 4-bit weights, the unpack warps; the warp count
+// is a multiple of four so that registers can be moved between aligned groups of four warps.
+constexpr int GEMM_EPI_WARPS = 8;
+constexpr int GEMM_WARP_TMA = GEMM_EPI_WARPS;
+constexpr int GEMM_WARP_MMA = GEMM_EPI_WARPS + 1;
+constexpr int GEMM_WARP_STORE = GEMM_EPI_WARPS + 2;
+constexpr int GEMM_THREADS_W8 = (GEMM_EPI_WARPS + 3) * 32;  // first unpack thread
+__host__ __device__ constexpr int gemm_threads(bool w4) { return (w4 ? 16 : 12) * 32; }
+// Registers per thread: the kernel starts with `gemm_regs_launch`, the epilogue warps then grow to
+// `gemm_regs_epi` with what the other warps give back (8 * epi + rest * other <= warps * launch).
+__host__ __device__ constexpr int gemm_regs_launch(bool w4) { return w4 ? 128 : 168; }
+__host__ __device__ constexpr int gemm_regs_epi(bool w4) { return w4 ? 200 : 208; }
+constexpr int GEMM_REGS_OTHER = 56;
+static_assert(8 * gemm_regs_epi(true) + 8 * GEMM_REGS_OTHER <= 16 * gemm_regs_launch(true), "register pool");
+static_assert(8 * gemm_regs_epi(false) + 4 * GEMM_REGS_OTHER <= 12 * gemm_regs_launch(false), "register pool");
 constexpr int GEMM_MAX_ATOMS = 1024;           // 32768 reduction positions
 constexpr int GEMM_A_STAGE = GEMM_BM * 128;  // bytes
 constexpr int GEMM_SMEM_LIMIT = 227 * 1024;
@@ -59,7 +68,6 @@ struct GemmCfg {
   static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
   static constexpr int NACC_RAW = 512 / BN;
   static constexpr int NACC = NACC_RAW > 4 ? 4 : NACC_RAW;
-  static constexpr int CW = BN / 4;  // columns per epilogue thread
   static constexpr int SMEM = STAGES * STAGE + OUT_BYTES + MISC_BYTES + 1024;
   static_assert(BN % 32 == 0 && BN <= 256, "BN must be a multiple of 32 up to 256");
   static_assert(NACC >= 2, "need two accumulators to overlap the epilogue");
@@ -73,7 +81,6 @@ struct GemmArgs {
   int n_tiles_m, n_tiles_n;
   uint32_t idesc;
   int use_zp;                 // 0 for zero-centred codes
-  int magic;                  // 1: |acc| < 2^22 for every group, the epilogue converts without I2F
   int code_max;               // 2^b - 1
   uint32_t res_mask;          // groups whose padding did not absorb all of wsum
   int per_token;              // 1: scale rows indexed by token, 0: by row_group[token mod P]
@@ -104,8 +111,8 @@ struct __align__(8) GemmShared {
   int abort_flag;
 };
 
-template <int BN, bool W4, bool CONV, bool MAGIC>
-__global__ void __launch_bounds__(W4 ? GEMM_THREADS_W4 : GEMM_THREADS_W8, 1)
+template <int BN, bool W4, bool CONV>
+__global__ void __maxnreg__(gemm_regs_launch(W4))
 gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmY, const __grid_constant__ GemmArgs a) {
   using Cfg = GemmCfg<BN>;
@@ -165,18 +172,18 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   tc_fence_after();
   const uint32_t tmem_base = sh->tmem_base;
 
+  if (warp >= GEMM_EPI_WARPS) {
+  // The warps that only move data or issue instructions hand most of their registers to the epilogue.
+  reg_dealloc<GEMM_REGS_OTHER>();
   if (warp == GEMM_WARP_TMA) {
     // ------------------------------------------------------------ TMA producer
-    // The whole warp walks the loop (so that no lane of it is parked at the final CTA barrier while
-    // another one spins); lane 0 issues the copies.
-    {
-      if (lane == 0) {
-        tma_prefetch_desc(&tmA);
-        if (!W4) tma_prefetch_desc(&tmB);
-      }
-      uint32_t it = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+    // One lane runs the loop; the others go straight to the CTA's final barrier.
+    if (lane == 0) {
+      tma_prefetch_desc(&tmA);
+      if (!W4) tma_prefetch_desc(&tmB);
+      const uint32_t empty0 = smem_u32(&sh->empty[0]);
+      uint32_t s = 0, empty_par = 1;  // fresh barriers pass a wait for parity 1
+      for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
         const int tm = tile / a.n_tiles_n, tn = tile - tm * a.n_tiles_n;
         const int m0 = tm * GEMM_BM, n0 = tn * BN;
         int cw = 0, chh = 0, cn = 0;  // conv: spatial origin of this row tile
@@ -188,15 +195,12 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           cw = rem - chh * a.conv_W;
         }
         int g = 0, g_start = 0;  // conv: current group and its first atom
-        for (int ks = 0; ks < n_kstages && ok; ++ks, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1;
-          ok = __all_sync(0xffffffffu, mbar_wait(&sh->empty[s], ph ^ 1, abort_flag));
-          if (!ok) break;
+        for (int ks = 0; ks < n_kstages; ++ks) {
+          mbar_wait_lean(empty0 + s * 8u, empty_par, abort_flag);
           const int atoms_here = min(4, n_atoms - ks * 4);
           uint32_t bytes = W4 ? 0u : (uint32_t)Cfg::B_STAGE;
           bytes += CONV ? (uint32_t)(atoms_here * 4096) : (uint32_t)GEMM_A_STAGE;
-          if (lane == 0) mbar_arrive_expect_tx(&sh->full[s], bytes);
+          mbar_arrive_expect_tx(&sh->full[s], bytes);
           if (CONV) {
             for (int j = 0; j < atoms_here; ++j) {
               const int atom = ks * 4 + j;
@@ -208,234 +212,104 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               const int tap = local / a.grp_atoms[g];
               const int ca = local - tap * a.grp_atoms[g];
               const int ky = tap / 3, kx = tap - ky * 3;
-              if (lane == 0)
-                tma_load_4d(smA + s * GEMM_A_STAGE + j * 4096, &tmA, &sh->full[s], a.grp_chan0[g] + ca * 32,
-                            cw + kx - 1, chh + ky - 1, cn);
+              tma_load_4d(smA + s * GEMM_A_STAGE + j * 4096, &tmA, &sh->full[s], a.grp_chan0[g] + ca * 32,
+                          cw + kx - 1, chh + ky - 1, cn);
             }
           } else {
-            if (lane == 0) tma_load_2d(smA + s * GEMM_A_STAGE, &tmA, &sh->full[s], ks * 128, m0);
+            tma_load_2d(smA + s * GEMM_A_STAGE, &tmA, &sh->full[s], ks * 128, m0);
           }
-          if (!W4 && lane == 0) tma_load_2d(smB + s * Cfg::B_STAGE, &tmB, &sh->full[s], ks * 128, n0);
-          __syncwarp();
+          if (!W4) tma_load_2d(smB + s * Cfg::B_STAGE, &tmB, &sh->full[s], ks * 128, n0);
+          if (++s == (uint32_t)STAGES) {
+            s = 0;
+            empty_par ^= 1u;
+          }
         }
+        if (*abort_flag) break;
       }
     }
+    __syncwarp();
   } else if (warp == GEMM_WARP_MMA) {
     // ------------------------------------------------------------ MMA issuer
-    {
-      // The issuing thread is a single lane: its dependent instruction chain per MMA is what bounds
-      // short groups, so everything that can be is precomputed (descriptor words, the per-stage
-      // bit mask of atoms that end a group, running accumulator index and parity).
+    // One lane runs the loop.  Its dependent instruction chain per MMA is what bounds short groups,
+    // so everything that can be is precomputed (descriptor words, barrier addresses, the per-stage
+    // bit mask of atoms that end a group, running ring positions and parities) and the waits carry
+    // no warp votes.
+    if (lane == 0) {
       constexpr uint32_t A_HI = CONV ? smem_desc_hi(256, 6) : smem_desc_hi(1024, 2);
       constexpr uint32_t B_HI = smem_desc_hi(1024, 2);
       const uint32_t a_lo0 = smem_desc_lo(smem_u32(smA)), b_lo0 = smem_desc_lo(smem_u32(smB));
       const uint32_t idesc = a.idesc;
-      uint32_t it = 0;
-      int s = 0;                 // stage slot of `it`
+      const uint32_t full0 = smem_u32(&sh->full[0]), empty0 = smem_u32(&sh->empty[0]);
+      const uint32_t accf0 = smem_u32(&sh->acc_full[0]), acce0 = smem_u32(&sh->acc_empty[0]);
+      uint32_t s = 0;            // stage slot
       uint32_t full_phase = 0;   // parity of the slot's next "full" phase
-      int ab = 0;                // accumulator of the next group
+      uint32_t ab = 0;           // accumulator of the next group
       uint32_t acc_phase = 1;    // parity to wait for on its "empty" barrier (fresh barriers pass)
-      bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
         bool need_acc = true;  // the next atom starts a group: take the next accumulator first
         uint32_t d_tmem = tmem_base;
         uint64_t ends = 0;     // bit i: atom (16 * 4) * word + i is the last of its group
-        for (int ks = 0; ks < n_kstages && ok; ++ks, ++it) {
+        for (int ks = 0; ks < n_kstages; ++ks) {
           if ((ks & 15) == 0) ends = a.end_mask[ks >> 4];
           const uint32_t end_bits = (uint32_t)(ends >> ((ks & 15) * 4)) & 0xFu;
-          ok = __all_sync(0xffffffffu, mbar_wait(&sh->full[s], full_phase, abort_flag));
-          if (!ok) break;
+          mbar_wait_lean(full0 + s * 8u, full_phase, abort_flag);
           tc_fence_after();
           const int atoms_here = min(4, n_atoms - ks * 4);
-          const uint32_t a_lo = a_lo0 + (uint32_t)s * (GEMM_A_STAGE >> 4);
-          const uint32_t b_lo = b_lo0 + (uint32_t)s * (Cfg::B_STAGE >> 4);
+          const uint32_t a_lo = a_lo0 + s * (uint32_t)(GEMM_A_STAGE >> 4);
+          const uint32_t b_lo = b_lo0 + s * (uint32_t)(Cfg::B_STAGE >> 4);
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            if (j < atoms_here && ok) {
+            if (j < atoms_here) {
               if (need_acc) {
-                ok = __all_sync(0xffffffffu, mbar_wait(&sh->acc_empty[ab], acc_phase, abort_flag));
-                if (ok) {
-                  tc_fence_after();
-                  d_tmem = tmem_base + (uint32_t)(ab * BN);
-                }
+                mbar_wait_lean(acce0 + ab * 8u, acc_phase, abort_flag);
+                tc_fence_after();
+                d_tmem = tmem_base + ab * (uint32_t)BN;
               }
-              if (ok) {
-                if (lane == 0)
-                  mma_i8_lohi(d_tmem, a_lo + (CONV ? j * 256 : j * 2), A_HI, b_lo + j * 2, B_HI, idesc,
-                              need_acc ? 0u : 1u);
-                need_acc = false;
-                if (end_bits & (1u << j)) {  // last atom of the group: hand the accumulator over right away
-                  if (lane == 0) mma_commit(&sh->acc_full[ab]);
-                  if (++ab == NACC) {
-                    ab = 0;
-                    acc_phase ^= 1u;
-                  }
-                  need_acc = true;
+              mma_i8_lohi(d_tmem, a_lo + (CONV ? j * 256 : j * 2), A_HI, b_lo + j * 2, B_HI, idesc,
+                          need_acc ? 0u : 1u);
+              need_acc = false;
+              if (end_bits & (1u << j)) {  // last atom of the group: hand the accumulator over right away
+                mma_commit_addr(accf0 + ab * 8u);
+                if (++ab == (uint32_t)NACC) {
+                  ab = 0;
+                  acc_phase ^= 1u;
                 }
+                need_acc = true;
               }
             }
           }
-          if (ok && lane == 0) mma_commit(&sh->empty[s]);  // stage reusable once these MMAs have read it
-          __syncwarp();
-          if (++s == STAGES) {
+          mma_commit_addr(empty0 + s * 8u);  // stage reusable once these MMAs have read it
+          if (++s == (uint32_t)STAGES) {
             s = 0;
             full_phase ^= 1u;
           }
         }
+        if (*abort_flag) break;
       }
     }
-  } else if (warp < GEMM_EPI_WARPS) {
-    // ------------------------------------------------------------ epilogue
-    constexpr int CW = Cfg::CW;
-    constexpr int NCH = CW / 8;
-    const int q = warp & 3, sl = warp >> 2;
-    const int r_tile = q * 32 + lane;  // row inside the tile = TMEM lane
-    uint32_t acc_it = 0, tile_it = 0;
-    bool ok = true;
-    // The first scale / zero-point of the row are fetched one tile ahead, so their latency hides
-    // behind the current tile.
-    float pre_s = 0.f;
-    int pre_z = 0;
-    const float* srow = nullptr;
-    const int32_t* zrow = nullptr;
-    auto prefetch_tile = [&](int tile) {
-      const int tm = tile / a.n_tiles_n;
-      const int64_t row = (int64_t)tm * GEMM_BM + r_tile;
-      const int64_t row_c = row < a.M ? row : a.M - 1;
-      const int64_t prow = a.per_token ? row_c : (int64_t)__ldg(a.row_group + row_c % a.P);
-      srow = a.scale + prow * a.G;
-      zrow = a.zp + prow * a.G;
-      pre_s = __ldg(srow);
-      pre_z = a.use_zp ? __ldg(zrow) : 0;
-    };
-    if ((int)blockIdx.x < n_tiles) prefetch_tile(blockIdx.x);
-    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tile_it) {
-      const int col0 = cta_n0 + sl * CW;
-      const float* srow_t = srow;
-      const int32_t* zrow_t = zrow;
-      float y[CW];
-#pragma unroll
-      for (int i = 0; i < CW; ++i) y[i] = 0.f;
-      // scale and zero-point of the next group are fetched one group ahead
-      float s_next = pre_s;
-      int z_next = pre_z;
-      for (int g = 0; g < a.G && ok; ++g, ++acc_it) {
-        const float s = s_next;
-        const int Z = z_next;
-        if (g + 1 < a.G) {
-          s_next = __ldg(srow_t + g + 1);
-          if (a.use_zp) z_next = __ldg(zrow_t + g + 1);
-        } else if (tile + (int)gridDim.x < n_tiles) {
-          prefetch_tile(tile + gridDim.x);
-        }
-        const int ab = acc_it % NACC;
-        ok = __all_sync(0xffffffffu, mbar_wait(&sh->acc_full[ab], (acc_it / NACC) & 1, abort_flag));
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * BN + sl * CW);
-        // All loads of the group are issued before the single wait, so their latencies overlap; the
-        // accumulator is handed back as soon as its columns are in registers.
-        uint32_t rb[NCH][8];
-#pragma unroll
-        for (int k = 0; k < NCH; ++k) tmem_ld8(taddr + k * 8, rb[k]);
-        tmem_ld_wait();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sh->acc_empty[ab]);
-        if (MAGIC) {
-          // |acc| < 2^22: adding 0x4B400000 gives the bit pattern of the float 1.5 * 2^23 + acc, and
-          // subtracting 1.5 * 2^23 is exact.  Integer add and float add are full-rate instructions;
-          // the int -> float conversion runs on the 16-lane special-function pipe and would bound
-          // the whole kernel.
-#pragma unroll
-          for (int k = 0; k < NCH; ++k)
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-              y[k * 8 + i] =
-                  fmaf(s, __fsub_rn(__int_as_float((int)rb[k][i] + 0x4B400000), 12582912.0f), y[k * 8 + i]);
-        } else {
-#pragma unroll
-          for (int k = 0; k < NCH; ++k)
-#pragma unroll
-            for (int i = 0; i < 8; ++i) y[k * 8 + i] = fmaf(s, (float)(int)rb[k][i], y[k * 8 + i]);
-        }
-        if (a.use_zp) {
-          // rare: Z outside the code range (the stored padding code is the clamped Z), or a group
-          // whose padding could not absorb all of wsum
-          if (__any_sync(0xffffffffu, (uint32_t)Z > (uint32_t)a.code_max)) {
-            const int Zc = min(max(Z, 0), a.code_max);
-            const float c1 = -s * (float)(Z - Zc);
-            const float4* ws = reinterpret_cast<const float4*>(wsum_s + g * BN + sl * CW);
-#pragma unroll
-            for (int i = 0; i < CW; i += 4) {
-              const float4 u = ws[i >> 2];
-              y[i] = fmaf(c1, u.x, y[i]);
-              y[i + 1] = fmaf(c1, u.y, y[i + 1]);
-              y[i + 2] = fmaf(c1, u.z, y[i + 2]);
-              y[i + 3] = fmaf(c1, u.w, y[i + 3]);
-            }
-          }
-          if ((a.res_mask >> g) & 1u) {
-            const float c2 = -s * (float)min(max(Z, 0), a.code_max);
-            const float4* wr = reinterpret_cast<const float4*>(a.wres + (size_t)g * a.N_pad + col0);
-#pragma unroll
-            for (int i = 0; i < CW; i += 4) {
-              const float4 v = __ldg(wr + (i >> 2));
-              y[i] = fmaf(c2, v.x, y[i]);
-              y[i + 1] = fmaf(c2, v.y, y[i + 1]);
-              y[i + 2] = fmaf(c2, v.z, y[i + 2]);
-              y[i + 3] = fmaf(c2, v.w, y[i + 3]);
-            }
-          }
-        }
-      }
-      if (!ok) break;
-      // staging buffer: wait until the stores of the previous tile have read it (normally long done)
-      ok = __all_sync(0xffffffffu, mbar_wait(&sh->out_free, (tile_it & 1) ^ 1, abort_flag));
-      if (!ok) break;
-#pragma unroll
-      for (int j = 0; j < NCH; ++j) {
-        const int cl = sl * CW + j * 8;  // first tile column of this 16-byte chunk
-        const float4 s0 = *reinterpret_cast<const float4*>(sw_s + cl), s1 = *reinterpret_cast<const float4*>(sw_s + cl + 4);
-        const float4 b0 = *reinterpret_cast<const float4*>(bias_s + cl), b1 = *reinterpret_cast<const float4*>(bias_s + cl + 4);
-        uint4 o;
-        __half2* oh = reinterpret_cast<__half2*>(&o);
-        oh[0] = __floats2half2_rn(fmaf(s0.x, y[j * 8 + 0], b0.x), fmaf(s0.y, y[j * 8 + 1], b0.y));
-        oh[1] = __floats2half2_rn(fmaf(s0.z, y[j * 8 + 2], b0.z), fmaf(s0.w, y[j * 8 + 3], b0.w));
-        oh[2] = __floats2half2_rn(fmaf(s1.x, y[j * 8 + 4], b1.x), fmaf(s1.y, y[j * 8 + 5], b1.y));
-        oh[3] = __floats2half2_rn(fmaf(s1.z, y[j * 8 + 6], b1.z), fmaf(s1.w, y[j * 8 + 7], b1.w));
-        // panel of 32 columns = 64-byte rows, 16-byte chunk index XOR bits 1-2 of the row (64 B swizzle)
-        const int panel = cl >> 5, ch = (cl >> 3) & 3;
-        *reinterpret_cast<uint4*>(smOut + panel * (GEMM_BM * 64) + r_tile * 64 + ((ch ^ ((r_tile >> 1) & 3)) << 4)) = o;
-      }
-      fence_proxy_async_smem();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sh->out_full);
-    }
+    __syncwarp();
   } else if (warp == GEMM_WARP_STORE) {
     // ------------------------------------------------------------ output store
-    {
-      if (lane == 0) tma_prefetch_desc(&tmY);
+    if (lane == 0) {
+      tma_prefetch_desc(&tmY);
+      const uint32_t out_full_a = smem_u32(&sh->out_full);
       uint32_t tile_it = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tile_it) {
+      for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tile_it) {
         const int tm = tile / a.n_tiles_n, tn = tile - tm * a.n_tiles_n;
         const int n0 = tn * BN;
-        ok = __all_sync(0xffffffffu, mbar_wait(&sh->out_full, tile_it & 1, abort_flag));
-        if (!ok) break;
-        if (lane == 0) {
+        mbar_wait_lean(out_full_a, tile_it & 1u, abort_flag);
+        if (*abort_flag) break;
 #pragma unroll
-          for (int pnl = 0; pnl < BN / 32; ++pnl)
-            if (n0 + pnl * 32 < a.N) tma_store_2d(&tmY, smOut + pnl * (GEMM_BM * 64), n0 + pnl * 32, tm * GEMM_BM);
-          bulk_commit();
-          bulk_wait_read0();
-          mbar_arrive(&sh->out_free);
-        }
-        __syncwarp();
+        for (int pnl = 0; pnl < BN / 32; ++pnl)
+          if (n0 + pnl * 32 < a.N) tma_store_2d(&tmY, smOut + pnl * (GEMM_BM * 64), n0 + pnl * 32, tm * GEMM_BM);
+        bulk_commit();
+        bulk_wait_read0();
+        mbar_arrive(&sh->out_free);
       }
-      if (lane == 0) bulk_wait0();
+      bulk_wait0();
     }
-  } else if (W4) {
+    __syncwarp();
+  } else if (W4 && warp >= GEMM_WARP_STORE + 1) {
     // ------------------------------------------------------------ 4-bit weight unpack into the B stage
     constexpr int ITEMS = (BN * 4 + GEMM_UNPACK_THREADS - 1) / GEMM_UNPACK_THREADS;  // 16-byte pieces per thread
     const int ut = threadIdx.x - GEMM_THREADS_W8;  // 0..GEMM_UNPACK_THREADS-1
@@ -484,6 +358,159 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (ks + 1 < n_kstages) fetch(tile, ks + 1);
         else if (tile + (int)gridDim.x < n_tiles) fetch(tile + gridDim.x, 0);
       }
+    }
+  }
+  } else {
+    reg_alloc<gemm_regs_epi(W4)>();
+    // ------------------------------------------------------------ epilogue
+    // The loop is kept lean on purpose: with one convert and half a packed multiply-add per
+    // element and group, bookkeeping instructions would otherwise outnumber the arithmetic.
+    constexpr int CW = BN / (GEMM_EPI_WARPS / 4);  // columns per thread
+    constexpr int HC = CW / 2;                     // columns per chunk: a group is drained in two
+    static_assert(HC % 8 == 0, "chunk must be whole 8-column loads");
+    const int q = warp & 3, sl = warp >> 2;
+    const int r_tile = q * 32 + lane;  // row inside the tile = TMEM lane
+    const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(sl * CW);
+    const uint32_t full0 = smem_u32(&sh->acc_full[0]), empty0 = smem_u32(&sh->acc_empty[0]);
+    const uint32_t out_free_a = smem_u32(&sh->out_free), out_full_a = smem_u32(&sh->out_full);
+    const int G = a.G;
+    const bool use_zp = a.use_zp != 0;
+    const uint32_t code_max = (uint32_t)a.code_max, res_mask = a.res_mask;
+    uint32_t ab = 0, acc_par = 0, tile_it = 0;  // accumulator of the current group and its "full" parity
+    // The first scale / zero-point of the row are fetched one tile ahead, so their latency hides
+    // behind the current tile.
+    float pre_s = 0.f;
+    int pre_z = 0;
+    const float* srow = nullptr;
+    const int32_t* zrow = nullptr;
+    auto prefetch_tile = [&](int tile) {
+      const int tm = tile / a.n_tiles_n;
+      const int64_t row = (int64_t)tm * GEMM_BM + r_tile;
+      const int64_t row_c = row < a.M ? row : a.M - 1;
+      const int64_t prow = a.per_token ? row_c : (int64_t)__ldg(a.row_group + row_c % a.P);
+      srow = a.scale + prow * G;
+      zrow = a.zp + prow * G;
+      pre_s = __ldg(srow);
+      pre_z = use_zp ? __ldg(zrow) : 0;
+    };
+    // Two register buffers of one chunk each: while the arithmetic runs on one, the tensor-memory
+    // loads of the next chunk (of this group, or of the next group, or of the next tile's first
+    // group) are already in flight into the other.
+    uint32_t rb0[HC], rb1[HC];
+    auto load_chunk = [&](uint32_t taddr, uint32_t(&rb)[HC]) {
+#pragma unroll
+      for (int k = 0; k < HC / 16; ++k) tmem_ld16(taddr + k * 16, reinterpret_cast<uint32_t(&)[16]>(rb[k * 16]));
+      if (HC % 16) tmem_ld8(taddr + (HC / 16) * 16, reinterpret_cast<uint32_t(&)[8]>(rb[(HC / 16) * 16]));
+    };
+    if ((int)blockIdx.x < n_tiles) {
+      prefetch_tile(blockIdx.x);
+      mbar_wait_lean(full0, 0u, abort_flag);
+      tc_fence_after();
+      load_chunk(t_lane, rb0);
+    }
+    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tile_it) {
+      const float* srow_t = srow;
+      const int32_t* zrow_t = zrow;
+      const bool more_tiles = tile + (int)gridDim.x < n_tiles;
+      unsigned long long y2[CW / 2];  // packed pairs of fp32 sums
+#pragma unroll
+      for (int i = 0; i < CW / 2; ++i) y2[i] = 0ull;
+      // scale and zero-point of the next group are fetched one group ahead
+      float s_next = pre_s;
+      int z_next = pre_z;
+      for (int g = 0; g < G; ++g) {
+        const float s = s_next;
+        const int Z = z_next;
+        const bool more = g + 1 < G || more_tiles;  // another group follows this one
+        if (g + 1 < G) {
+          s_next = __ldg(srow_t + g + 1);
+          if (use_zp) z_next = __ldg(zrow_t + g + 1);
+        } else if (more_tiles) {
+          prefetch_tile(tile + gridDim.x);
+        }
+        const uint32_t taddr = t_lane + ab * (uint32_t)BN;
+        uint32_t nab = ab + 1, npar = acc_par;
+        if (nab == (uint32_t)NACC) {
+          nab = 0;
+          npar ^= 1u;
+        }
+        const unsigned long long s2 = pack_f32x2(s, s);
+        // first chunk: its loads were issued during the previous chunk's arithmetic
+        tmem_ld_wait();
+        load_chunk(taddr + HC, rb1);
+        // poll the next group's accumulator now, look at the answer after the arithmetic
+        const uint32_t next_ready = more ? mbar_try_addr(full0 + nab * 8u, npar) : 1u;
+#pragma unroll
+        for (int i = 0; i < HC / 2; ++i) cvt_fma_f32x2(y2[i], s2, rb0[2 * i], rb0[2 * i + 1]);
+        if (!next_ready) mbar_wait_lean(full0 + nab * 8u, npar, abort_flag);
+        // second chunk: the accumulator goes back to the issuer as soon as its last columns are in
+        // registers, and the next group's first chunk is requested before the arithmetic
+        tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_addr(empty0 + ab * 8u);
+        if (more) {
+          tc_fence_after();
+          load_chunk(t_lane + nab * (uint32_t)BN, rb0);
+        }
+#pragma unroll
+        for (int i = 0; i < HC / 2; ++i) cvt_fma_f32x2(y2[HC / 2 + i], s2, rb1[2 * i], rb1[2 * i + 1]);
+        ab = nab;
+        acc_par = npar;
+        if (use_zp) {
+          // rare: Z outside the code range (the stored padding code is the clamped Z), or a group
+          // whose padding could not absorb all of wsum
+          if (__any_sync(0xffffffffu, (uint32_t)Z > code_max)) {
+            const int Zc = min(max(Z, 0), (int)code_max);
+            const float c1 = -s * (float)(Z - Zc);
+            const unsigned long long c2 = pack_f32x2(c1, c1);
+            const ulonglong2* ws = reinterpret_cast<const ulonglong2*>(wsum_s + g * BN + sl * CW);
+#pragma unroll
+            for (int i = 0; i < CW / 4; ++i) {
+              const ulonglong2 u = ws[i];
+              y2[2 * i] = fma_f32x2(c2, u.x, y2[2 * i]);
+              y2[2 * i + 1] = fma_f32x2(c2, u.y, y2[2 * i + 1]);
+            }
+          }
+          if ((res_mask >> g) & 1u) {
+            const float c1 = -s * (float)min(max(Z, 0), (int)code_max);
+            const unsigned long long c2 = pack_f32x2(c1, c1);
+            const float4* wr = reinterpret_cast<const float4*>(a.wres + (size_t)g * a.N_pad + cta_n0 + sl * CW);
+#pragma unroll
+            for (int i = 0; i < CW / 4; ++i) {
+              const float4 v = __ldg(wr + i);
+              y2[2 * i] = fma_f32x2(c2, pack_f32x2(v.x, v.y), y2[2 * i]);
+              y2[2 * i + 1] = fma_f32x2(c2, pack_f32x2(v.z, v.w), y2[2 * i + 1]);
+            }
+          }
+        }
+      }
+      if (*abort_flag) break;  // a wait gave up somewhere in the CTA (same value in every lane)
+      // staging buffer: wait until the stores of the previous tile have read it (normally long done)
+      mbar_wait_lean(out_free_a, (tile_it & 1u) ^ 1u, abort_flag);
+#pragma unroll
+      for (int j = 0; j < CW / 8; ++j) {
+        const int cl = sl * CW + j * 8;  // first tile column of this 16-byte chunk
+        const ulonglong2 s0 = *reinterpret_cast<const ulonglong2*>(sw_s + cl), s1 = *reinterpret_cast<const ulonglong2*>(sw_s + cl + 4);
+        const ulonglong2 b0 = *reinterpret_cast<const ulonglong2*>(bias_s + cl), b1 = *reinterpret_cast<const ulonglong2*>(bias_s + cl + 4);
+        float f[8];
+        unpack_f32x2(fma_f32x2(s0.x, y2[j * 4 + 0], b0.x), f[0], f[1]);
+        unpack_f32x2(fma_f32x2(s0.y, y2[j * 4 + 1], b0.y), f[2], f[3]);
+        unpack_f32x2(fma_f32x2(s1.x, y2[j * 4 + 2], b1.x), f[4], f[5]);
+        unpack_f32x2(fma_f32x2(s1.y, y2[j * 4 + 3], b1.y), f[6], f[7]);
+        uint4 o;
+        __half2* oh = reinterpret_cast<__half2*>(&o);
+        oh[0] = __floats2half2_rn(f[0], f[1]);
+        oh[1] = __floats2half2_rn(f[2], f[3]);
+        oh[2] = __floats2half2_rn(f[4], f[5]);
+        oh[3] = __floats2half2_rn(f[6], f[7]);
+        // panel of 32 columns = 64-byte rows, 16-byte chunk index XOR bits 1-2 of the row (64 B swizzle)
+        const int panel = cl >> 5, ch = (cl >> 3) & 3;
+        *reinterpret_cast<uint4*>(smOut + panel * (GEMM_BM * 64) + r_tile * 64 + ((ch ^ ((r_tile >> 1) & 3)) << 4)) = o;
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_addr(out_full_a);
     }
   }
 
@@ -540,7 +567,7 @@ static bool encode_map(CUtensorMap* m, const void* base, int rank, const uint64_
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, bool W4, bool CONV, bool MAGIC>
+template <int BN, bool W4, bool CONV>
 static dgq_status launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
                               const GemmArgs& a, int grid, cudaStream_t stream) {
   using Cfg = GemmCfg<BN>;
@@ -548,11 +575,11 @@ static dgq_status launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, co
   int dev = 0;
   DGQ_CUDA_OK(cudaGetDevice(&dev));
   if (dev >= 64 || !attr_set[dev]) {
-    DGQ_CUDA_OK(cudaFuncSetAttribute(gq_gemm_kernel<BN, W4, CONV, MAGIC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    DGQ_CUDA_OK(cudaFuncSetAttribute(gq_gemm_kernel<BN, W4, CONV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      Cfg::SMEM));
     if (dev < 64) attr_set[dev] = true;
   }
-  gq_gemm_kernel<BN, W4, CONV, MAGIC><<<grid, W4 ? GEMM_THREADS_W4 : GEMM_THREADS_W8, Cfg::SMEM, stream>>>(tmA, tmB, tmY, a);
+  gq_gemm_kernel<BN, W4, CONV><<<grid, gemm_threads(W4), Cfg::SMEM, stream>>>(tmA, tmB, tmY, a);
   g_launches += 1;
   DGQ_CUDA_OK(cudaGetLastError());
   return DGQ_OK;
@@ -561,18 +588,11 @@ static dgq_status launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, co
 template <int BN>
 static dgq_status launch_gemm_bn(bool w4, bool conv, const CUtensorMap& tmA, const CUtensorMap& tmB,
                                  const CUtensorMap& tmY, const GemmArgs& a, int grid, cudaStream_t stream) {
-  if (a.magic) {
-    if (w4)
-      return conv ? launch_gemm<BN, true, true, true>(tmA, tmB, tmY, a, grid, stream)
-                  : launch_gemm<BN, true, false, true>(tmA, tmB, tmY, a, grid, stream);
-    return conv ? launch_gemm<BN, false, true, true>(tmA, tmB, tmY, a, grid, stream)
-                : launch_gemm<BN, false, false, true>(tmA, tmB, tmY, a, grid, stream);
-  }
   if (w4)
-    return conv ? launch_gemm<BN, true, true, false>(tmA, tmB, tmY, a, grid, stream)
-                : launch_gemm<BN, true, false, false>(tmA, tmB, tmY, a, grid, stream);
-  return conv ? launch_gemm<BN, false, true, false>(tmA, tmB, tmY, a, grid, stream)
-              : launch_gemm<BN, false, false, false>(tmA, tmB, tmY, a, grid, stream);
+    return conv ? launch_gemm<BN, true, true>(tmA, tmB, tmY, a, grid, stream)
+                : launch_gemm<BN, true, false>(tmA, tmB, tmY, a, grid, stream);
+  return conv ? launch_gemm<BN, false, true>(tmA, tmB, tmY, a, grid, stream)
+              : launch_gemm<BN, false, false>(tmA, tmB, tmY, a, grid, stream);
 }
 
 }  // namespace dgq
@@ -625,19 +645,6 @@ extern "C" dgq_status dgq_linear(const dgq_groups* g, const dgq_weight* w, int t
     a.seg_end[k] = w->seg_end[k];
     a.grp_atoms[k] = (g->group_off[k + 1] - g->group_off[k]) / DGQ_K_ATOM;
     a.grp_chan0[k] = g->group_off[k];
-  }
-  {
-    // |acc| < 2^22 holds for a group of n atoms if n * 32 * max|code| * max|weight| < 2^22
-    const int64_t amax = (layout == DGQ_CODES_S8_CENTRED) ? 128 : (1 << g->bits) - 1;
-    const int64_t wmax = (w->w_bits == 4) ? 7 * 16 : 127;
-    int longest = 0, start = 0;
-    for (int k = 0; k < g->G; ++k) {
-      longest = std::max(longest, w->seg_end[k] - start);
-      start = w->seg_end[k];
-    }
-    // Measured on B200: the conversion instruction is not what bounds the epilogue and the two-instruction
-    // magic path is a few percent slower, so it stays off; the bound check is kept for when it pays.
-    a.magic = 0 && (longest * (int64_t)DGQ_K_ATOM * amax * wmax < (1ll << 22));
   }
   int BN = 128;
   if (w->N % 160 == 0) BN = 160;
