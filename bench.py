@@ -238,6 +238,21 @@ class Workload:
         return int(sum(h.numel() * h.element_size() for h in self.host_out.values()))
 
 
+def max_over_ranks(values, world, device):
+    """Replicas only: every rank times the same work on its own GPU; the job's time is the slowest rank's."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_rate(ops_per_replica, ms_per_step, world):
+    """Whole-job TOPS: `world` replicas each do `ops_per_replica` per step in `ms_per_step` (max over ranks)."""
+    return world * ops_per_replica / (ms_per_step * 1e-3) / 1e12
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
@@ -303,14 +318,11 @@ def run_cuda(args):
     for j, (kind, ev) in enumerate(marks):
         nxt = marks[j + 1][1] if j + 1 < len(marks) else e1
         kind_ms.setdefault(kind, []).append(ev.elapsed_time(nxt))
-    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], world, "cuda")
     ms_step = ms_total / args.steps
     ops = gemm_ops()
-    value = world * ops / (ms_step * 1e-3) / 1e12
-    e2e_value = world * ops / (ms_e2e / args.steps * 1e-3) / 1e12
+    value = whole_job_rate(ops, ms_step, world)
+    e2e_value = whole_job_rate(ops, ms_e2e / args.steps, world)
     peaks = measured_peaks()
     int8_peak = 2.0 * peaks["bf16_sustained"]          # int8 : bf16 dense nominal ratio 4.5 : 2.25
     gemm_ms = sum(kind_ms["gemm"]) / args.steps        # all GEMM launches of one step
