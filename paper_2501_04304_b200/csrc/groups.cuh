@@ -19,6 +19,7 @@ struct dgq_groups {
   // device copies
   int16_t* d_perm = nullptr;          // [K_pad], -1 = padding
   uint8_t* d_chunk_group = nullptr;   // [K_pad / 16] group of every 16-code chunk
+  uint8_t* d_quant_head = nullptr;    // layout tables of the quantizer, as it keeps them in shared memory
   int32_t* d_row_group = nullptr;     // [P]
   int32_t* d_col_group = nullptr;     // [C]
   float* d_scale = nullptr;           // [T][R][G]
@@ -228,6 +229,7 @@ constexpr int GROUP_MIN_PAD = 8;
 static void groups_free_device(dgq_groups* g) {
   cudaFree(g->d_perm);
   cudaFree(g->d_chunk_group);
+  cudaFree(g->d_quant_head);
   cudaFree(g->d_row_group);
   cudaFree(g->d_col_group);
   cudaFree(g->d_scale);
@@ -239,6 +241,14 @@ static void groups_free_device(dgq_groups* g) {
 // group padded to a multiple of DGQ_K_ATOM positions with at least GROUP_MIN_PAD padding positions.
 // The padding carries the cell's zero-point as its code; the weight side stores -wsum spread over
 // those positions, so the integer product already contains the zero-point term of Eq. 1.
+// The quantizer's layout tables: position of every channel in the group-contiguous order (int16 [C]),
+// group of every 16-code chunk (u8 [K_pad / 16]) and the padding positions of every chunk as a bit
+// mask (u16 [K_pad / 16], 2-byte aligned), in one block whose size is a multiple of 16 bytes.
+__host__ __device__ inline int quant_head_pm_offset(int C, int K_pad) { return (C * 2 + (K_pad >> 4) + 1) & ~1; }
+__host__ __device__ inline int quant_head_bytes(int C, int K_pad) {
+  return (quant_head_pm_offset(C, K_pad) + (K_pad >> 4) * 2 + 15) & ~15;
+}
+
 static dgq_status groups_build_layout(dgq_groups* g) {
   g->group_off.assign(g->G + 1, 0);
   g->perm.clear();
@@ -267,6 +277,18 @@ static dgq_status groups_build_layout(dgq_groups* g) {
   DGQ_CUDA_OK(cudaMalloc(&g->d_zp, tn * sizeof(int32_t)));
   DGQ_CUDA_OK(cudaMemcpy(g->d_perm, perm16.data(), g->K_pad * sizeof(int16_t), cudaMemcpyHostToDevice));
   DGQ_CUDA_OK(cudaMemcpy(g->d_chunk_group, cg.data(), cg.size(), cudaMemcpyHostToDevice));
+  {
+    std::vector<uint8_t> head(quant_head_bytes(g->C, g->K_pad), 0);
+    int16_t* pos = reinterpret_cast<int16_t*>(head.data());
+    uint16_t* pm = reinterpret_cast<uint16_t*>(head.data() + quant_head_pm_offset(g->C, g->K_pad));
+    for (int p = 0; p < g->K_pad; ++p) {
+      if (g->perm[p] >= 0) pos[g->perm[p]] = (int16_t)p;
+      else pm[p >> 4] |= (uint16_t)(1u << (p & 15));
+    }
+    std::memcpy(head.data() + g->C * 2, cg.data(), cg.size());
+    DGQ_CUDA_OK(cudaMalloc(&g->d_quant_head, head.size()));
+    DGQ_CUDA_OK(cudaMemcpy(g->d_quant_head, head.data(), head.size(), cudaMemcpyHostToDevice));
+  }
   DGQ_CUDA_OK(cudaMemcpy(g->d_row_group, g->row_group.data(), g->P * sizeof(int32_t), cudaMemcpyHostToDevice));
   DGQ_CUDA_OK(cudaMemcpy(g->d_col_group, g->col_group.data(), g->C * sizeof(int32_t), cudaMemcpyHostToDevice));
   return DGQ_OK;

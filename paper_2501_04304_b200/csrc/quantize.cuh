@@ -1,14 +1,16 @@
 // Activation quantizer: Eq. 1 with the per-cell parameters of Eq. 6, fused with the channel
 // permutation into the padded, group-contiguous code layout the GEMM reads.
 //
-// One warp owns one or two rows at a time and never synchronises with the rest of the CTA: it
-// stages its rows in shared memory with coalesced 128-bit loads, then every lane takes 16-code
-// chunks of the output (all 16 codes of a chunk belong to one channel group, since groups are
-// padded to multiples of 32 positions), gathers their source channels through the permutation
-// table and writes one 16-byte vector, so a warp writes 512 contiguous bytes.
-// Dynamic-token mode first reduces the range of every (row, group) cell: a lane reduces its
-// chunks, lanes that share a cell merge through shared-memory atomics on order-preserving
-// integer keys, and one lane per cell derives (s, 1/s, Z).
+// One warp owns one or two rows at a time and never synchronises with the rest of the CTA.  It
+// loads its rows with coalesced 128-bit loads and scatters every value to its position in the
+// group-contiguous order inside a shared-memory row buffer (padding positions of the buffer hold
+// NaN for good).  After that every 16-code chunk of the output is 32 contiguous bytes of the
+// buffer that belong to one channel group: a lane reads a chunk with two 128-bit loads, reduces
+// its range with packed half-precision min / max (which skip NaN), converts, quantizes and writes
+// one 16-byte vector, so a warp writes 512 contiguous bytes.
+// Dynamic-token mode first reduces the range of every (row, group) cell: lanes that share a cell
+// merge through shared-memory atomics on order-preserving integer keys, and one lane per cell
+// derives (s, 1/s, Z).
 // HBM traffic: 2 B read + 1 B written per element (+ 8 B per (token, group) in dynamic mode).
 #pragma once
 
@@ -25,8 +27,7 @@ struct QuantArgs {
   int64_t M, ld;
   int C, K_pad, G, P, bits, rows_per_warp;
   int dynamic, centred;
-  const int16_t* perm;
-  const uint8_t* chunk_group;
+  const uint8_t* head;     // layout tables (see quant_head_bytes)
   const int32_t* row_group;
   const float* inv_scale;  // static: table row of the timestep [R][G]
   const int32_t* zp;
@@ -34,39 +35,37 @@ struct QuantArgs {
   int32_t* dyn_zp;
 };
 
-// The 16 source channels of one chunk (two 128-bit loads of int16 indices; -1 = padding).
-__device__ __forceinline__ void load_chunk_perm(const int16_t* perm, int ch, int (&c)[16]) {
-  const uint4 lo = *reinterpret_cast<const uint4*>(perm + ch * 16);
-  const uint4 hi = *(reinterpret_cast<const uint4*>(perm + ch * 16) + 1);
-  const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    c[2 * j] = (int)(int16_t)(w[j] & 0xFFFFu);
-    c[2 * j + 1] = (int)(int16_t)(w[j] >> 16);
-  }
+__host__ __device__ inline int qa_warp_bytes(int rpw, int K_pad, int G) { return rpw * K_pad * 2 + rpw * G * 16; }
+
+// bits 0-3 of `m` spread to 0xFF bytes
+__device__ __forceinline__ uint32_t nibble_to_byte_mask(uint32_t m) {
+  return (((m & 0xFu) * 0x00204081u) & 0x01010101u) * 0xFFu;
 }
 
 __global__ void __launch_bounds__(QA_THREADS, 4) quantize_act_kernel(const QuantArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int n_chunks = a.K_pad >> 4;
-  // layout: perm [K_pad] int16 | chunk_group [n_chunks] u8 | per warp: rows [rpw][C] fp16, cells [rpw][G] x 4 ints
-  int16_t* perm_s = reinterpret_cast<int16_t*>(smem_raw);
-  uint8_t* cg_s = reinterpret_cast<uint8_t*>(perm_s + a.K_pad);
-  const int head = (a.K_pad * 2 + n_chunks + 15) & ~15;
+  int16_t* pos_s = reinterpret_cast<int16_t*>(smem_raw);             // position of every channel
+  uint8_t* cg_s = reinterpret_cast<uint8_t*>(pos_s + a.C);            // group of every chunk
+  uint16_t* pm_s = reinterpret_cast<uint16_t*>(smem_raw + quant_head_pm_offset(a.C, a.K_pad));  // padding positions of every chunk
+  const int head = quant_head_bytes(a.C, a.K_pad);
   const int rpw = a.rows_per_warp;
-  const int warp_bytes = ((rpw * a.C * 2 + 15) & ~15) + rpw * a.G * 16;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  unsigned char* wbase = smem_raw + head + warp * warp_bytes;
-  __half* rows_s = reinterpret_cast<__half*>(wbase);
-  int* cell_lo = reinterpret_cast<int*>(wbase + ((rpw * a.C * 2 + 15) & ~15));
+  unsigned char* wbase = smem_raw + head + warp * qa_warp_bytes(rpw, a.K_pad, a.G);
+  __half* rows_s = reinterpret_cast<__half*>(wbase);                  // [rpw][K_pad], group-contiguous order
+  int* cell_lo = reinterpret_cast<int*>(wbase + rpw * a.K_pad * 2);
   int* cell_hi = cell_lo + rpw * a.G;
   float* cell_inv = reinterpret_cast<float*>(cell_hi + rpw * a.G);
   int* cell_z = reinterpret_cast<int*>(cell_inv + rpw * a.G);
 
-  for (int i = threadIdx.x; i < a.K_pad / 8; i += QA_THREADS)
-    reinterpret_cast<uint4*>(perm_s)[i] = __ldg(reinterpret_cast<const uint4*>(a.perm) + i);
-  for (int i = threadIdx.x; i < n_chunks; i += QA_THREADS) cg_s[i] = a.chunk_group[i];
+  for (int i = threadIdx.x; i < head / 16; i += QA_THREADS)
+    reinterpret_cast<uint4*>(smem_raw)[i] = __ldg(reinterpret_cast<const uint4*>(a.head) + i);
   __syncthreads();
+  // The row buffers start as NaN everywhere: every row overwrites the positions of its channels, the
+  // padding positions are never written again.
+  for (int i = lane; i < rpw * a.K_pad / 8; i += 32)
+    reinterpret_cast<uint4*>(rows_s)[i] = make_uint4(0x7FFF7FFFu, 0x7FFF7FFFu, 0x7FFF7FFFu, 0x7FFF7FFFu);
+  __syncwarp();
 
   const int vec_per_row = a.C >> 3;
   const float Lf = (float)((1 << a.bits) - 1);
@@ -77,20 +76,33 @@ __global__ void __launch_bounds__(QA_THREADS, 4) quantize_act_kernel(const Quant
     // the first store, so the memory latency is paid once per batch and not once per piece.
     {
       const int n_vec = rows * vec_per_row;
+      const uint4* xrow = reinterpret_cast<const uint4*>(a.X + row0 * a.ld);
+      const int64_t row_step = a.ld >> 3;  // in 128-bit pieces
+      uint16_t* dst0 = reinterpret_cast<uint16_t*>(rows_s);
       for (int v0 = 0; v0 < n_vec; v0 += 4 * 32) {
         uint4 x[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const int i = v0 + e * 32 + lane;
           if (i < n_vec) {
-            const int r = i / vec_per_row, v = i - r * vec_per_row;
-            x[e] = __ldg(reinterpret_cast<const uint4*>(a.X + (row0 + r) * a.ld) + v);
+            const int r = i >= vec_per_row ? 1 : 0, v = i - r * vec_per_row;  // at most two rows per warp
+            x[e] = __ldg(xrow + r * row_step + v);
           }
         }
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const int i = v0 + e * 32 + lane;
-          if (i < n_vec) reinterpret_cast<uint4*>(rows_s)[i] = x[e];  // rows are packed: pitch C halfs
+          if (i < n_vec) {
+            const int r = i >= vec_per_row ? 1 : 0, v = i - r * vec_per_row;
+            const uint4 pp = *reinterpret_cast<const uint4*>(pos_s + v * 8);  // positions of these 8 channels
+            uint16_t* dst = dst0 + r * a.K_pad;
+            const uint32_t pw[4] = {pp.x, pp.y, pp.z, pp.w}, xw[4] = {x[e].x, x[e].y, x[e].z, x[e].w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              dst[pw[j] & 0xFFFFu] = (uint16_t)(xw[j] & 0xFFFFu);
+              dst[pw[j] >> 16] = (uint16_t)(xw[j] >> 16);
+            }
+          }
         }
       }
     }
@@ -103,19 +115,19 @@ __global__ void __launch_bounds__(QA_THREADS, 4) quantize_act_kernel(const Quant
 
     if (a.dynamic) {
       for (int r = 0; r < rows; ++r) {
-        const __half* row = rows_s + r * a.C;
+        const uint4* row = reinterpret_cast<const uint4*>(rows_s + r * a.K_pad);
         for (int ch = lane; ch < n_chunks; ch += 32) {
-          float lo = INFINITY, hi = -INFINITY;
-          int cidx[16];
-          load_chunk_perm(perm_s, ch, cidx);
-#pragma unroll
-          for (int j = 0; j < 16; ++j)
-            if (cidx[j] >= 0) {
-              const float v = __half2float(row[cidx[j]]);
-              lo = fminf(lo, v);
-              hi = fmaxf(hi, v);
-            }
-          if (lo <= hi) {
+          const uint4 u0 = row[ch * 2], u1 = row[ch * 2 + 1];
+          const __half2* h0 = reinterpret_cast<const __half2*>(&u0);
+          const __half2* h1 = reinterpret_cast<const __half2*>(&u1);
+          // NaN (padding, or a NaN input) never wins a min / max
+          __half2 lo2 = __hmin2(__hmin2(__hmin2(h0[0], h0[1]), __hmin2(h0[2], h0[3])),
+                                __hmin2(__hmin2(h1[0], h1[1]), __hmin2(h1[2], h1[3])));
+          __half2 hi2 = __hmax2(__hmax2(__hmax2(h0[0], h0[1]), __hmax2(h0[2], h0[3])),
+                                __hmax2(__hmax2(h1[0], h1[1]), __hmax2(h1[2], h1[3])));
+          const float lo = __half2float(__hmin(__low2half(lo2), __high2half(lo2)));
+          const float hi = __half2float(__hmax(__low2half(hi2), __high2half(hi2)));
+          if (lo <= hi) {  // false when the whole chunk is padding
             const int g = cg_s[ch];
             atomicMin(&cell_lo[r * a.G + g], float_to_ordered(lo));
             atomicMax(&cell_hi[r * a.G + g], float_to_ordered(hi));
@@ -142,7 +154,7 @@ __global__ void __launch_bounds__(QA_THREADS, 4) quantize_act_kernel(const Quant
     }
 
     for (int r = 0; r < rows; ++r) {
-      const __half* row = rows_s + r * a.C;
+      const uint4* row = reinterpret_cast<const uint4*>(rows_s + r * a.K_pad);
       const int rg = a.dynamic ? 0 : a.row_group[(row0 + r) % a.P];
       uint8_t* out = a.Xq + (row0 + r) * a.K_pad;
       for (int ch = lane; ch < n_chunks; ch += 32) {
@@ -157,22 +169,49 @@ __global__ void __launch_bounds__(QA_THREADS, 4) quantize_act_kernel(const Quant
           Z = __ldg(a.zp + rg * a.G + g);
         }
         const float Zf = (float)Z;
-        const int pad_code = a.centred ? 0 : min(max(Z, 0), (1 << a.bits) - 1);
         const int sub = a.centred ? Z : 0;
+        const uint4 u[2] = {row[ch * 2], row[ch * 2 + 1]};
+        const __half2* h = reinterpret_cast<const __half2*>(u);
         uint32_t w[4];
-        int cidx[16];
-        load_chunk_perm(perm_s, ch, cidx);
+        if (abs(Z) <= (1 << 21)) {
+          // Eq. 1 without conversion instructions, bit-identical to quantize_code for |Z| <= 2^21:
+          // t + 1.5 * 2^23 rounds t to the nearest-even integer (|t| < 2^22; a larger |t| ends at a
+          // clamp either way), subtracting (1.5 * 2^23 - Z) is exact and leaves rint(t) + Z, NaN
+          // falls to 0 in fmaxf, and after the clamps the code is the low byte of (q + 1.5 * 2^23).
+          const float MAGIC = 12582912.0f;
+          const float mz = MAGIC - Zf, ms = MAGIC - (float)sub;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          uint32_t word = 0;
+          for (int q = 0; q < 4; ++q) {
+            const float2 f0 = __half22float2(h[2 * q]), f1 = __half22float2(h[2 * q + 1]);
+            const float fv[4] = {f0.x, f0.y, f1.x, f1.y};
+            uint32_t b[4];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int c = cidx[q * 4 + j];
-            int code = pad_code;
-            if (c >= 0) code = quantize_code(__half2float(row[c]), inv_s, Zf, Lf) - sub;
-            word |= (uint32_t)(code & 0xFF) << (8 * j);
+            for (int j = 0; j < 4; ++j) {
+              float v = __fsub_rn(__fadd_rn(__fmul_rn(fv[j], inv_s), MAGIC), mz);
+              v = fminf(fmaxf(v, 0.0f), Lf);
+              b[j] = __float_as_uint(__fadd_rn(v, ms));  // low byte = code - sub (two's complement)
+            }
+            w[q] = __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
           }
-          w[q] = word;
+        } else {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const float2 f0 = __half22float2(h[2 * q]), f1 = __half22float2(h[2 * q + 1]);
+            const int c0 = quantize_code(f0.x, inv_s, Zf, Lf) - sub, c1 = quantize_code(f0.y, inv_s, Zf, Lf) - sub;
+            const int c2 = quantize_code(f1.x, inv_s, Zf, Lf) - sub, c3 = quantize_code(f1.y, inv_s, Zf, Lf) - sub;
+            w[q] = (uint32_t)(c0 & 0xFF) | ((uint32_t)(c1 & 0xFF) << 8) | ((uint32_t)(c2 & 0xFF) << 16) |
+                   ((uint32_t)c3 << 24);
+          }
+        }
+        const uint32_t pm = pm_s[ch];
+        if (pm) {  // padding positions carry the clamped zero-point (0 in the zero-centred layout)
+          const uint32_t pad_code = a.centred ? 0u : (uint32_t)min(max(Z, 0), (1 << a.bits) - 1);
+          const uint32_t padw = pad_code * 0x01010101u;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint32_t m = nibble_to_byte_mask(pm >> (4 * q));
+            w[q] = (w[q] & ~m) | (padw & m);
+          }
         }
         *reinterpret_cast<uint4*>(out + ch * 16) = make_uint4(w[0], w[1], w[2], w[3]);
       }
@@ -216,19 +255,15 @@ extern "C" dgq_status dgq_quantize_act(const dgq_groups* g, int timestep, int mo
   a.bits = g->bits;
   a.dynamic = (mode == DGQ_MODE_DYNAMIC_TOKEN);
   a.centred = (layout == DGQ_CODES_S8_CENTRED);
-  a.perm = g->d_perm;
-  a.chunk_group = g->d_chunk_group;
+  a.head = g->d_quant_head;
   a.row_group = g->d_row_group;
   a.inv_scale = g->d_inv_scale + trow;
   a.zp = g->d_zp + trow;
   a.dyn_scale = dyn_scale;
   a.dyn_zp = dyn_zp;
-  const int n_chunks = g->K_pad / 16;
   const int rpw = (g->C <= 1280) ? 2 : 1;
   a.rows_per_warp = rpw;
-  const int head = (g->K_pad * 2 + n_chunks + 15) & ~15;
-  const int warp_bytes = ((rpw * g->C * 2 + 15) & ~15) + rpw * g->G * 16;
-  const size_t smem = (size_t)head + (size_t)QA_WARPS * warp_bytes;
+  const size_t smem = (size_t)quant_head_bytes(g->C, g->K_pad) + (size_t)QA_WARPS * qa_warp_bytes(rpw, g->K_pad, g->G);
   if (smem > 200 * 1024) return DGQ_ERR_UNSUPPORTED;
   static bool attr_set[64] = {false};
   int dev = 0;
