@@ -1,0 +1,92 @@
+"""GPU parity at the sizes and launch configurations the benchmark times (persistent kernels, several tiles
+per CTA, every SM busy): outputs are checked on sampled rows that the oracle computes one by one."""
+import numpy as np
+import pytest
+
+from oracle import calibration as oc
+from oracle import linear as ol
+from paper_2501_04304_b200 import synth
+from dgq_testlib import gpu, to_dev, unpermute_codes
+from test_gpu_attention import _compare
+
+pytestmark = pytest.mark.gpu
+
+REL = 1e-3
+
+
+def _sample_rows(M, seed):
+    rng = np.random.default_rng(seed)
+    fixed = [0, 1, 127, 128, 129, 255, 256, M // 2 - 1, M // 2, M - 129, M - 128, M - 2, M - 1]
+    rows = np.unique(np.concatenate([np.asarray(fixed), rng.integers(0, M, 64)]))
+    return rows[(rows >= 0) & (rows < M)]
+
+
+@pytest.mark.parametrize("P,batch,C,N,w_bits", [
+    (4096, 2, 320, 2560, 8),     # FF1 of the 64 x 64 level: 64 x 16 tiles on 144 CTAs
+    (4096, 2, 1280, 320, 8),     # FF2: long K, two column blocks
+    (4096, 2, 320, 960, 8),      # stacked q/k/v projection
+    (1024, 8, 640, 640, 4),      # 32 x 32 level, 4-bit weights
+])
+def test_linear_full_size_sampled_rows(P, batch, C, N, w_bits):
+    torch, b = gpu()
+    M = P * batch
+    Xcal = synth.activations(21, 100, 4, P, C)
+    X = synth.activations(21, 1, batch, P, C)
+    W = synth.weights(21, 2, N, C)
+    bias = synth.bias(21, 3, N)
+    gr = oc.calibrate(Xcal, P, 8, 8, dim_select=oc.DIM_CHANNEL)
+    g = b.calibrate_groups(to_dev(torch, Xcal), P, 8, 8, b.DIM_CHANNEL)
+    wq, sw = ol.weight_rtn(W, w_bits)
+    w = b.weight_prepare(g, to_dev(torch, W), w_bits)
+    Xq, ds, dz = b.quantize_act(g, to_dev(torch, X), mode=b.MODE_DYNAMIC_TOKEN)
+    Y = b.linear(g, w, Xq, mode=b.MODE_DYNAMIC_TOKEN, dyn_scale=ds, dyn_zp=dz, bias=to_dev(torch, bias))
+    torch.cuda.synchronize()
+    assert b.device_status() == 0
+    rows = _sample_rows(M, 5)
+    codes, s_rows, z_rows = ol.quantize_dynamic_token(X[rows], gr.col_group, gr.G, gr.bits)
+    got_codes = unpermute_codes(Xq[torch.from_numpy(rows).cuda()], g.export()["perm"], C)
+    assert np.array_equal(got_codes, codes)                      # integer work: bit-exact
+    Yref = ol.group_linear(codes, s_rows, z_rows, gr.col_group, wq, sw, bias)
+    Yg = Y[torch.from_numpy(rows).cuda()].float().cpu().numpy().astype(np.float64)
+    err = np.max(np.abs(Yg - Yref))
+    assert err <= REL * np.max(np.abs(Yref)), f"max|delta| {err:.3e} on sampled rows"
+    assert np.isfinite(Y.float().cpu().numpy()).all()            # every tile was written
+
+
+def test_conv_full_size_sampled_bands():
+    """2 x 64 x 64 x 320 -> 320, W4A6, 16 groups: image-border and interior bands of output rows."""
+    torch, b = gpu()
+    n, H, Wd, C, N, K = 2, 64, 64, 320, 320, 16
+    P = H * Wd
+    Xcal = synth.activations(22, 100, 4, P, C, None, None, token_outliers=False)
+    X = synth.activations(22, 1, n, P, C, None, None, token_outliers=False)
+    Wt = synth.conv_weights(22, 2, N, C)
+    bias = synth.bias(22, 3, N)
+    gr = oc.calibrate(Xcal, P, 6, K, dim_select=oc.DIM_CHANNEL)
+    g = b.calibrate_groups(to_dev(torch, Xcal), P, 6, K, b.DIM_CHANNEL)
+    wq, sw = ol.weight_rtn(Wt, 4)
+    conv = (n, H, Wd, C)
+    w = b.weight_prepare(g, to_dev(torch, Wt), 4, conv=conv)
+    Xq, _, _ = b.quantize_act(g, to_dev(torch, X), layout=b.CODES_S8_CENTRED)
+    Y = b.linear(g, w, Xq, layout=b.CODES_S8_CENTRED, bias=to_dev(torch, bias), conv=conv)
+    torch.cuda.synchronize()
+    assert b.device_status() == 0
+    Yg = Y.float().cpu().numpy().astype(np.float64).reshape(n, H, Wd, N)
+    codes, _, _ = ol.quantize_static(X, gr, 0)
+    codes = codes.reshape(n, H, Wd, C)
+    worst, ref_max = 0.0, 0.0
+    for img, h0, h1 in [(0, 0, 2), (0, 31, 33), (0, 62, 64), (1, 0, 1), (1, 1, 3), (1, 63, 64)]:
+        lo, hi = max(h0 - 1, 0), min(h1 + 1, H)                  # the band with the rows it reads
+        sub = ol.group_conv3x3(codes[img:img + 1, lo:hi], gr.scale[0][0], gr.zp[0][0], gr.col_group, wq, sw, bias)
+        ref = sub[0, h0 - lo:h0 - lo + (h1 - h0)]                # rows whose neighbours are real rows or the border
+        worst = max(worst, np.max(np.abs(Yg[img, h0:h1] - ref)))
+        ref_max = max(ref_max, np.max(np.abs(ref)))
+    assert worst <= REL * ref_max, f"max|delta| {worst:.3e} vs max|ref| {ref_max:.3e}"
+    assert np.isfinite(Yg).all()
+
+
+def test_attention_full_size():
+    """B 2, H 8, nq 4096, nk 77, d 40, 8-bit codes: the whole output against the oracle."""
+    torch, b = gpu()
+    Q, K, V = synth.attention_inputs(23, 2, 8, 4096, 77, 40)
+    _compare(torch, b, Q, K, V, 8)
