@@ -5,11 +5,12 @@
 // (Eq. 1's de-quantizer with the group parameters of Eq. 6) fused in.
 //
 // CTA = one 128-row output tile x BN columns, persistent over tiles.  Warp roles:
-//   warps 0-15  epilogue: lane quarter = warp & 3 (the TMEM lanes a warp may read), column slice = warp >> 2
-//   warp  16    TMA producer (one elected lane): A code tile and B weight tile per 128-byte K stage
-//   warp  17    MMA issuer (one elected lane) and TMEM allocator
-//   warp  18    output store (one elected lane): TMA stores of the staged fp16 tile
-//   warps 19-21 (4-bit weights only) unpack packed nibbles from global memory into the B stage
+//   warps 0-7   epilogue: lane quarter = warp & 3 (the TMEM lanes a warp may read), column half = warp >> 2
+//   warp  8     TMA producer (one lane): A code tile and B weight tile per 128-byte K stage
+//   warp  9     MMA issuer (one lane) and TMEM allocator
+//   warp  10    output store (one lane): TMA stores of the staged fp16 tile
+//   warps 11-15 (4-bit weights only) unpack packed nibbles from global memory into the B stage
+// After set-up the data-movement warps hand registers to the epilogue warps (setmaxnreg).
 // K runs over 32-code atoms; a stage holds four atoms.  Group segments are multiples of one atom,
 // so the issuer moves to the next TMEM accumulator between two atoms, commits the finished one to
 // the epilogue and keeps going while the epilogue drains it.
