@@ -253,6 +253,26 @@ def whole_job_rate(ops_per_replica, ms_per_step, world):
     return world * ops_per_replica / (ms_per_step * 1e-3) / 1e12
 
 
+# DRAM bytes (read + written) of the six GEMM launches of one step, from one ncu capture of this
+# benchmark (profiles/gq_gemm_kernel_bench_step_dram.md).  Valid only for the kernel sources it was
+# taken with: any change to them turns the figure back into null.
+GEMM_DRAM_BYTES_PER_STEP = 41_147_136
+GEMM_SOURCES = ("paper_2501_04304_b200/csrc/linear.cuh", "paper_2501_04304_b200/csrc/common.cuh")
+GEMM_SOURCES_SHA1 = "61c1b3cc14fb3a7dc993762655c2548f4ed059ab"
+
+
+def gemm_traffic():
+    import hashlib
+    h = hashlib.sha1()
+    try:
+        for f in GEMM_SOURCES:
+            with open(os.path.join(ROOT, f), "rb") as fh:
+                h.update(fh.read())
+    except OSError:
+        return None
+    return GEMM_DRAM_BYTES_PER_STEP if h.hexdigest() == GEMM_SOURCES_SHA1 else None
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
@@ -342,7 +362,8 @@ def run_cuda(args):
                 "d2h_bytes_per_step": wl.d2h_bytes(), "ms_per_step": ms_e2e / args.steps},
         "gpu_launches": int(launches),
         "roofline": {"bound": "tensor", "achieved": gemm_tops, "peak": int8_peak, "unit": "TOP/s",
-                     "frac": gemm_tops / int8_peak, "traffic": None,
+                     "frac": gemm_tops / int8_peak, "traffic": gemm_traffic(),
+                     "traffic_unit": "DRAM bytes per step over the 6 launches (ncu); outputs are still in L2 when a launch ends",
                      "kernel": "gq_gemm_kernel (6 launches per step, timed as one CUDA graph)",
                      "peak_source": f"2 x bf16 sustained, {peaks['source']}"},
         "kernels": {
