@@ -64,7 +64,7 @@ struct GemmCfg {
   static constexpr int B_STAGE = BN * 128;
   static constexpr int STAGE = GEMM_A_STAGE + B_STAGE;
   static constexpr int OUT_BYTES = GEMM_BM * BN * 2;  // fp16 staging of one output tile
-  static constexpr int MISC_BYTES = 2048 + (2 + DGQ_MAX_GROUPS) * BN * 4;  // barriers + sw, bias, wsum of the CTA's columns
+  static constexpr int MISC_BYTES = 2048 + (2 + DGQ_MAX_GROUPS) * BN * 4 + GEMM_MAX_ATOMS * 4;  // barriers + sw, bias, wsum of the CTA's columns + conv atom table
   static constexpr int STAGES_RAW = (GEMM_SMEM_LIMIT - 1024 - OUT_BYTES - MISC_BYTES) / STAGE;
   static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
   static constexpr int NACC_RAW = 512 / BN;
@@ -131,6 +131,7 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   float* sw_s = reinterpret_cast<float*>(smOut + Cfg::OUT_BYTES + 2048);  // [BN]
   float* bias_s = sw_s + BN;                                              // [BN]
   float* wsum_s = bias_s + BN;                                            // [G][BN]
+  uint32_t* conv_tab = reinterpret_cast<uint32_t*>(wsum_s + DGQ_MAX_GROUPS * BN);  // [atoms] conv: channel | kx << 16 | ky << 18
   const int cta_n0 = ((int)blockIdx.x % a.n_tiles_n) * BN;
   volatile int* abort_flag = &sh->abort_flag;
 
@@ -164,6 +165,22 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int g = i / BN, c = i - g * BN;
       wsum_s[i] = cta_n0 + c < a.N_pad ? __ldg(a.wsum + (size_t)g * a.N_pad + cta_n0 + c) : 0.f;
     }
+  if (CONV) {
+    // Where every A atom of a tile comes from (same for all tiles): first channel position and
+    // filter tap.  Built once by all threads, so that the producer lane's chain per copy stays short.
+    for (int atom = threadIdx.x; atom < n_atoms; atom += blockDim.x) {
+      int g = 0, g_start = 0;
+      while (atom >= a.seg_end[g]) {
+        g_start = a.seg_end[g];
+        ++g;
+      }
+      const int local = atom - g_start;
+      const int tap = local / a.grp_atoms[g];
+      const int ca = local - tap * a.grp_atoms[g];
+      const int ky = tap / 3, kx = tap - ky * 3;
+      conv_tab[atom] = (uint32_t)(a.grp_chan0[g] + ca * 32) | ((uint32_t)kx << 16) | ((uint32_t)ky << 18);
+    }
+  }
   if (warp == GEMM_WARP_MMA) {
     tmem_alloc(&sh->tmem_base, 512);
     tmem_relinquish();
@@ -195,7 +212,6 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           chh = rem / a.conv_W;
           cw = rem - chh * a.conv_W;
         }
-        int g = 0, g_start = 0;  // conv: current group and its first atom
         for (int ks = 0; ks < n_kstages; ++ks) {
           mbar_wait_lean(empty0 + s * 8u, empty_par, abort_flag);
           const int atoms_here = min(4, n_atoms - ks * 4);
@@ -204,17 +220,9 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           mbar_arrive_expect_tx(&sh->full[s], bytes);
           if (CONV) {
             for (int j = 0; j < atoms_here; ++j) {
-              const int atom = ks * 4 + j;
-              while (atom >= a.seg_end[g]) {
-                g_start = a.seg_end[g];
-                ++g;
-              }
-              const int local = atom - g_start;
-              const int tap = local / a.grp_atoms[g];
-              const int ca = local - tap * a.grp_atoms[g];
-              const int ky = tap / 3, kx = tap - ky * 3;
-              tma_load_4d(smA + s * GEMM_A_STAGE + j * 4096, &tmA, &sh->full[s], a.grp_chan0[g] + ca * 32,
-                          cw + kx - 1, chh + ky - 1, cn);
+              const uint32_t e = conv_tab[ks * 4 + j];
+              tma_load_4d(smA + s * GEMM_A_STAGE + j * 4096, &tmA, &sh->full[s], (int)(e & 0xFFFFu),
+                          cw + (int)((e >> 16) & 3u) - 1, chh + (int)((e >> 18) & 3u) - 1, cn);
             }
           } else {
             tma_load_2d(smA + s * GEMM_A_STAGE, &tmA, &sh->full[s], ks * 128, m0);
