@@ -338,7 +338,19 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           pk[e] = __ldg(reinterpret_cast<const uint4*>(a.w_packed + (size_t)(n0 + r) * row_bytes + kb));
       }
     };
-    if ((int)blockIdx.x < n_tiles) fetch(blockIdx.x, 0);
+    // The CTA's whole column block of packed weights (BN rows of Kt / 2 bytes) is asked into L2 up
+    // front: the register look-ahead below is one stage deep, which covers an L2 hit but not a
+    // trip to DRAM.
+    if ((int)blockIdx.x < n_tiles) {
+      const int n0 = ((int)blockIdx.x % a.n_tiles_n) * BN;
+      const int lines_per_row = (row_bytes + 127) >> 7;
+      for (int i = ut; i < BN * lines_per_row; i += GEMM_UNPACK_THREADS) {
+        const int r = i / lines_per_row, l = i - r * lines_per_row;
+        const uint8_t* ptr = a.w_packed + (size_t)(n0 + r) * row_bytes + (size_t)l * 128;
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+      }
+      fetch(blockIdx.x, 0);
+    }
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
       for (int ks = 0; ks < n_kstages && ok; ++ks, ++it) {
         const int s = it % STAGES;
