@@ -190,6 +190,8 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_phase1_kernel(const AttnAr
   const int rows_valid = min(Cfg::WROWS, a.nq - row0);
   const int64_t q_stride = (int64_t)a.H * D;
   __half* slab = sQ + warp * Cfg::WROWS * Cfg::LDK;
+  pdl_launch_dependents();
+  pdl_wait();  // Q, K, V (and, in the second pass, the first pass's statistics) may come from earlier kernels
   uint4 xk[KStage<D, NKP>::N];
   load_k<D, NKP>(a, b, h, xk);
   if (rows_valid > 0) stage_q<D, NKP>(a.Q + (((int64_t)b * a.nq + row0) * a.H + h) * D, q_stride, rows_valid, slab);
@@ -261,6 +263,8 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_phase2_kernel(const AttnAr
   const int rows_valid = min(Cfg::WROWS, a.nq - row0);
   const int64_t q_stride = (int64_t)a.H * D;
   __half* slab = sQ + warp * Cfg::WROWS * Cfg::LDK;
+  pdl_launch_dependents();
+  pdl_wait();  // Q, K, V (and, in the second pass, the first pass's statistics) may come from earlier kernels
   uint4 xk[KStage<D, NKP>::N];
   load_k<D, NKP>(a, b, h, xk);
   // V^T: 128-bit loads of 8 features of one key, written transposed; keys >= nk and key 0 are zero.
@@ -403,11 +407,11 @@ static dgq_status launch_attn(const AttnArgs& a, cudaStream_t stream) {
   AttnArgs aa = a;
   aa.n_row_blocks = (a.nq + Cfg::ROWS - 1) / Cfg::ROWS;
   const int grid = a.B * a.H * aa.n_row_blocks;
-  attn_phase1_kernel<D, NKP><<<grid, AT_THREADS, SM1, stream>>>(aa);
+  DGQ_CUDA_OK(launch_pdl(attn_phase1_kernel<D, NKP>, dim3(grid), dim3(AT_THREADS), (size_t)SM1, stream, aa));
   if (a.codes_out)
-    attn_phase2_kernel<D, NKP, true><<<grid, AT_THREADS, SM2, stream>>>(aa);
+    DGQ_CUDA_OK(launch_pdl(attn_phase2_kernel<D, NKP, true>, dim3(grid), dim3(AT_THREADS), (size_t)SM2, stream, aa));
   else
-    attn_phase2_kernel<D, NKP, false><<<grid, AT_THREADS, SM2, stream>>>(aa);
+    DGQ_CUDA_OK(launch_pdl(attn_phase2_kernel<D, NKP, false>, dim3(grid), dim3(AT_THREADS), (size_t)SM2, stream, aa));
   g_launches += 2;
   DGQ_CUDA_OK(cudaGetLastError());
   return DGQ_OK;

@@ -8,7 +8,9 @@
 
 #include <atomic>
 #include <cstdint>
+#include <cstdlib>
 #include <cstring>
+#include <utility>
 #include <vector>
 
 #include "../../include/dgq.h"
@@ -74,12 +76,49 @@ __host__ __device__ __forceinline__ void group_params(float lo, float hi, int bi
 #endif
 }
 
+// Launch with the programmatic-serialization attribute (see pdl_wait); DGQ_PDL=0 in the environment
+// turns the attribute off.
+inline bool pdl_enabled() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = std::getenv("DGQ_PDL");
+    v = (e && e[0] == '0') ? 0 : 1;
+  }
+  return v != 0;
+}
+#ifdef __CUDACC__
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+#endif
 #ifdef __CUDACC__
 // Eq. 1: q = min(max(rint(x * inv_s) + Z, 0), L); NaN -> 0 (fmaxf returns the non-NaN operand).
 __device__ __forceinline__ int quantize_code(float x, float inv_s, float Zf, float Lf) {
   float u = __fadd_rn(rintf(__fmul_rn(x, inv_s)), Zf);
   return __float2int_rn(fminf(fmaxf(u, 0.0f), Lf));
 }
+
+// ------------------------------------------------------------------ programmatic dependent launch
+// Kernels of the hot path are launched so that the next kernel in the stream may be scheduled while
+// the current one drains (its blocks become resident as this one's exit, without the launch gap):
+// every such kernel calls pdl_launch_dependents() at its top and pdl_wait() before its first access
+// to global memory that an earlier kernel may have written.  pdl_wait() returns once every
+// preceding kernel has completed and its writes are visible; without the launch attribute both
+// are no-ops.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // ------------------------------------------------------------------ shared-memory addresses
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {

@@ -135,6 +135,7 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int cta_n0 = ((int)blockIdx.x % a.n_tiles_n) * BN;
   volatile int* abort_flag = &sh->abort_flag;
 
+  pdl_launch_dependents();
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int n_atoms = a.Kt >> 5;
@@ -185,6 +186,9 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     tmem_alloc(&sh->tmem_base, 512);
     tmem_relinquish();
   }
+  // Everything above reads only the layer's constants; codes, scales and zero-points may come from
+  // the kernel before this one.
+  pdl_wait();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -600,7 +604,8 @@ static dgq_status launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, co
                                      Cfg::SMEM));
     if (dev < 64) attr_set[dev] = true;
   }
-  gq_gemm_kernel<BN, W4, CONV><<<grid, gemm_threads(W4), Cfg::SMEM, stream>>>(tmA, tmB, tmY, a);
+  DGQ_CUDA_OK(launch_pdl(gq_gemm_kernel<BN, W4, CONV>, dim3(grid), dim3(gemm_threads(W4)), (size_t)Cfg::SMEM, stream, tmA,
+                         tmB, tmY, a));
   g_launches += 1;
   DGQ_CUDA_OK(cudaGetLastError());
   return DGQ_OK;

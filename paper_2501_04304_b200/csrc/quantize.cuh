@@ -58,8 +58,10 @@ __global__ void __launch_bounds__(QA_THREADS, 4) quantize_act_kernel(const Quant
   float* cell_inv = reinterpret_cast<float*>(cell_hi + rpw * a.G);
   int* cell_z = reinterpret_cast<int*>(cell_inv + rpw * a.G);
 
+  pdl_launch_dependents();
   for (int i = threadIdx.x; i < head / 16; i += QA_THREADS)
     reinterpret_cast<uint4*>(smem_raw)[i] = __ldg(reinterpret_cast<const uint4*>(a.head) + i);
+  pdl_wait();  // the layout tables above are constants of the grouping; the rows may come from the previous kernel
   __syncthreads();
   // The row buffers start as NaN everywhere: every row overwrites the positions of its channels, the
   // padding positions are never written again.
@@ -274,7 +276,7 @@ extern "C" dgq_status dgq_quantize_act(const dgq_groups* g, int timestep, int mo
   }
   const int64_t n_ctas = (M + (int64_t)QA_WARPS * rpw - 1) / ((int64_t)QA_WARPS * rpw);
   const int grid = (int)std::min<int64_t>(n_ctas, 148 * 8);
-  quantize_act_kernel<<<grid, QA_THREADS, smem, (cudaStream_t)stream>>>(a);
+  DGQ_CUDA_OK(launch_pdl(quantize_act_kernel, dim3(grid), dim3(QA_THREADS), smem, (cudaStream_t)stream, a));
   g_launches += 1;
   DGQ_CUDA_OK(cudaGetLastError());
   return DGQ_OK;

@@ -90,3 +90,61 @@ def test_attention_full_size():
     torch, b = gpu()
     Q, K, V = synth.attention_inputs(23, 2, 8, 4096, 77, 40)
     _compare(torch, b, Q, K, V, 8)
+
+
+def test_chained_layers_in_a_graph_match_serialised_calls():
+    """Back-to-back dependent kernels (quantize -> linear -> quantize -> linear -> attention on the result)
+    replayed as one CUDA graph give bit for bit what the same calls give with a device synchronisation after
+    each: the kernels are launched so that a kernel may be scheduled while its predecessor drains, and each
+    must wait for its predecessor's writes before it reads or writes anything."""
+    torch, b = gpu()
+    P, batch, C = 4096, 2, 320
+    M = P * batch
+    Xcal = synth.activations(31, 100, 4, P, C)
+    X = to_dev(torch, synth.activations(31, 1, batch, P, C))
+    g = b.calibrate_groups(to_dev(torch, Xcal), P, 8, 8, b.DIM_CHANNEL)
+    w1 = b.weight_prepare(g, to_dev(torch, synth.weights(31, 2, C, C)), 8)
+    w2 = b.weight_prepare(g, to_dev(torch, synth.weights(31, 3, C, C)), 8)
+    B, H, nq, nk, d = 2, 8, 4096, 77, 40
+    _, Kc, Vc = synth.attention_inputs(31, B, H, nq, nk, d)
+    Kd, Vd = to_dev(torch, Kc), to_dev(torch, Vc)
+
+    def buffers():
+        return dict(xq=torch.empty((M, g.K_pad), dtype=torch.uint8, device="cuda"),
+                    ds=torch.empty((M, g.G), dtype=torch.float32, device="cuda"),
+                    dz=torch.empty((M, g.G), dtype=torch.int32, device="cuda"),
+                    y1=torch.empty((M, C), dtype=torch.float16, device="cuda"),
+                    y2=torch.empty((M, C), dtype=torch.float16, device="cuda"),
+                    o=torch.empty((B, nq, H, d), dtype=torch.float16, device="cuda"),
+                    ws=torch.empty(b.cross_attn_workspace_bytes(B, H, nq, nk, d), dtype=torch.uint8, device="cuda"))
+
+    def chain(t, sync):
+        def s():
+            if sync:
+                torch.cuda.synchronize()
+        b.quantize_act_into(g, X, t["xq"], t["ds"], t["dz"], mode=b.MODE_DYNAMIC_TOKEN); s()
+        b.linear(g, w1, t["xq"], mode=b.MODE_DYNAMIC_TOKEN, dyn_scale=t["ds"], dyn_zp=t["dz"], out=t["y1"]); s()
+        b.quantize_act_into(g, t["y1"], t["xq"], t["ds"], t["dz"], mode=b.MODE_DYNAMIC_TOKEN); s()   # reuses the buffers
+        b.linear(g, w2, t["xq"], mode=b.MODE_DYNAMIC_TOKEN, dyn_scale=t["ds"], dyn_zp=t["dz"], out=t["y2"]); s()
+        q = t["y2"].view(B, nq, H, d)                                                                  # 8192 x 320
+        b.cross_attn_logq(q, Kd, Vd, 8, out=t["o"], workspace=t["ws"]); s()
+
+    ref = buffers()
+    chain(ref, sync=True)
+    torch.cuda.synchronize()
+    got = buffers()
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        chain(got, sync=False)                       # warm-up outside the capture
+        stream.synchronize()
+        for v in got.values():
+            v.zero_()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            chain(got, sync=False)
+        for _ in range(3):
+            graph.replay()
+    torch.cuda.synchronize()
+    assert b.device_status() == 0
+    for k in ("y1", "y2", "o"):
+        assert torch.equal(got[k], ref[k]), k
