@@ -196,11 +196,18 @@ class Workload:
             self.launch_kind(kind, i)
 
     def capture(self):
-        """One CUDA graph per (buffer set, kind): launch overhead stays out of the timed region."""
+        """Per buffer set: one CUDA graph of the whole step (what `value` is timed on) and one graph per
+        kind (what the per-kernel split is timed on); launch overhead stays out of the timed regions."""
         torch = self.torch
-        self.graphs, self.stream = [], torch.cuda.Stream()
-        n0 = self.b.launch_count()
+        self.graphs, self.step_graphs, self.stream = [], [], torch.cuda.Stream()
         with torch.cuda.stream(self.stream):
+            n0 = self.b.launch_count()
+            for i in range(self.n_sets):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=self.stream):
+                    self.step(i)
+                self.step_graphs.append(g)
+            self.launches_per_step = (self.b.launch_count() - n0) // self.n_sets
             for i in range(self.n_sets):
                 gs = {}
                 for kind in self.KINDS:
@@ -210,7 +217,9 @@ class Workload:
                     gs[kind] = g
                 self.graphs.append(gs)
         torch.cuda.synchronize()
-        self.launches_per_step = (self.b.launch_count() - n0) // self.n_sets
+
+    def replay_whole_step(self, i):
+        self.step_graphs[i % self.n_sets].replay()
 
     def replay_step(self, i, marks=None):
         gs = self.graphs[i % self.n_sets]
@@ -226,7 +235,7 @@ class Workload:
         s = self.sets[i % self.n_sets]
         for k, h in self.host.items():
             s["in"][k].copy_(h, non_blocking=True)
-        self.replay_step(i)
+        self.replay_whole_step(i)
         self.host_out["ff2"].copy_(s["out"]["ff2"], non_blocking=True)
         self.host_out["conv"].copy_(s["conv_out"], non_blocking=True)
         self.host_out["attn"].copy_(s["attn_out"], non_blocking=True)
@@ -303,20 +312,29 @@ def run_cuda(args):
     barrier()
     wl.capture()
     for i in range(max(args.warmup, 3)):
+        wl.replay_whole_step(i)
         wl.replay_step(i)
     barrier()
     sampler = ClockSampler(local)
     sampler.start()
-    marks = []
+    # timed region: K whole steps, one graph replay each
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record()
     for i in range(args.steps):
-        wl.replay_step(i, marks)
+        wl.replay_whole_step(i)
     e1.record()
     barrier()
     launches = wl.launches_per_step * args.steps
     ms_total = e0.elapsed_time(e1)
+    # the same K steps again, one graph per kind with an event in between, for the per-kernel split
+    marks = []
+    k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    k0.record()
+    for i in range(args.steps):
+        wl.replay_step(i, marks)
+    k1.record()
+    barrier()
     # end to end: host buffers in, results out, every step
     for i in range(2):
         wl.step_e2e(i)
@@ -336,7 +354,7 @@ def run_cuda(args):
     # duration of a kind = from its mark to the next mark (or to the end of the timed region)
     kind_ms = {}
     for j, (kind, ev) in enumerate(marks):
-        nxt = marks[j + 1][1] if j + 1 < len(marks) else e1
+        nxt = marks[j + 1][1] if j + 1 < len(marks) else k1
         kind_ms.setdefault(kind, []).append(ev.elapsed_time(nxt))
     ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], world, "cuda")
     ms_step = ms_total / args.steps
