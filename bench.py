@@ -74,37 +74,53 @@ def measured_peaks():
 
 
 class ClockSampler(threading.Thread):
-    """Samples nvidia-smi SM clocks and throttle reasons while the timed region runs."""
+    """Samples SM clocks and throttle reasons with ONE long-running `nvidia-smi -lms` child, started before
+    the warm-up so that no process is spawned while a timed region runs; `mark()` opens the window whose
+    samples are reported."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, index):
         super().__init__(daemon=True)
-        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
-        self._stop_evt = threading.Event()
+        self.index, self.rows, self.t_mark, self.proc = index, [], None, None
 
     def run(self):
-        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        while not self._stop_evt.is_set():
-            try:
-                out = subprocess.run(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-i",
-                                      str(self.index)], capture_output=True, text=True, timeout=5).stdout
-                f = [x.strip() for x in out.strip().split(",")]
-                self.samples.append(float(f[0]))
-                self.max_mhz = float(f[1])
-                for n, v in zip(names, f[2:]):
-                    if v.lower().startswith("active"):
-                        self.reasons.add(n)
-            except Exception:
-                pass
-            self._stop_evt.wait(0.1)
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "50"], stdout=subprocess.PIPE, text=True)
+            for line in self.proc.stdout:
+                f = [x.strip() for x in line.strip().split(",")]
+                if len(f) >= 6:
+                    self.rows.append((time.monotonic(), f))
+        except Exception:
+            pass
+
+    def mark(self):
+        self.t_mark = time.monotonic()
 
     def stop(self):
-        self._stop_evt.set()
-        self.join(timeout=10)
-        med = float(np.median(self.samples)) if self.samples else None
-        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(self.samples)}
+        if self.proc is not None:
+            self.proc.terminate()      # the exact child this object started
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+        self.join(timeout=5)
+        rows = [f for t, f in self.rows if self.t_mark is None or t >= self.t_mark] or [f for _, f in self.rows[-1:]]
+        mhz, reasons, max_mhz = [], set(), None
+        for f in rows:
+            try:
+                mhz.append(float(f[0]))
+                max_mhz = float(f[1])
+            except ValueError:
+                continue
+            for n, v in zip(self.NAMES, f[2:]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(mhz)) if mhz else None, "sm_max_mhz": max_mhz, "reasons": sorted(reasons),
+                "samples": len(mhz)}
 
 
 # ------------------------------------------------------------------------------------------ CUDA arm
@@ -307,6 +323,8 @@ def run_cuda(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local)
+    sampler.start()
     for i in range(3):
         wl.step(i)
     barrier()
@@ -315,8 +333,7 @@ def run_cuda(args):
         wl.replay_whole_step(i)
         wl.replay_step(i)
     barrier()
-    sampler = ClockSampler(local)
-    sampler.start()
+    sampler.mark()
     # timed region: K whole steps, one graph replay each
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
