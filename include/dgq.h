@@ -20,6 +20,12 @@
  *    `stream`; they allocate nothing and do not synchronise.  The calibration
  *    and weight-preparation calls allocate library-owned objects and
  *    synchronise with the host.
+ *  - The kernels these three calls enqueue are launched so that the next kernel
+ *    on the stream may be scheduled while the current one finishes; each waits
+ *    for everything enqueued before it on the stream before it reads or writes
+ *    memory, so stream order is kept as with ordinary launches, also inside a
+ *    captured CUDA graph.  Setting DGQ_PDL=0 in the environment before the
+ *    first call falls back to ordinary launches.
  *  - Device-side waits are bounded.  A kernel that gives up on a wait records
  *    DGQ_ERR_TIMEOUT in a device status word read by dgq_device_status().
  */
