@@ -6,7 +6,7 @@ from __future__ import annotations
 
 import numpy as np
 
-from .quantizers import log_quantize, log_dequantize
+from .quantizers import log_quantize, log_dequantize, group_params_array, quantize_canonical_f32
 
 PER_PROMPT, PER_PROMPT_HEAD, PER_CALL = 0, 1, 2
 FLT_MIN = float(np.finfo(np.float32).tiny)
@@ -42,7 +42,27 @@ def prompt_scale(A, gran=PER_PROMPT):
     return np.maximum(s, FLT_MIN)
 
 
-def cross_attn_logq(Q, K, V, bits, gran=PER_PROMPT, fixed_scale=None):
+def quantize_values(V, v_bits):
+    """V_hat of Eq. 9 when the value operand is quantized too.
+
+    The paper names V_hat "quantized value" without giving its quantizer; reading (parity unpinned): the
+    linear quantizer of Eq. 1 with the range of Eq. 6 taken over one head's [n_k, d] slab of one prompt,
+    code decided in fp32 (`quantize_canonical_f32`), de-quantized as s (q - Z) in fp32.  Rows j >= 1 are
+    the fp16 operand of the product and are rounded to fp16; row 0 (the <start> value, which meets a
+    full-precision score) stays fp32.  V [B, nk, H, d] -> (V_hat fp64 [B, nk, H, d], codes, s [B, H], Z [B, H]).
+    """
+    V32 = np.asarray(V, dtype=np.float32)
+    lo = V32.min(axis=(1, 3))
+    hi = V32.max(axis=(1, 3))
+    s, inv_s, Z = group_params_array(lo, hi, v_bits)                          # [B, H]
+    codes = quantize_canonical_f32(V32, inv_s[:, None, :, None], Z[:, None, :, None], v_bits)
+    deq = (s[:, None, :, None] * (codes - Z[:, None, :, None]).astype(np.float32)).astype(np.float32)
+    V_hat = deq.astype(np.float64)
+    V_hat[:, 1:] = deq[:, 1:].astype(np.float16).astype(np.float64)
+    return V_hat, codes, s, Z
+
+
+def cross_attn_logq(Q, K, V, bits, gran=PER_PROMPT, fixed_scale=None, v_bits=None):
     """Attention-aware quantization (Eq. 8, Eq. 9), fp64 throughout.
 
     Steps in the paper's order: full-precision softmax (Eq. 3); scale s from the
@@ -50,12 +70,13 @@ def cross_attn_logq(Q, K, V, bits, gran=PER_PROMPT, fixed_scale=None):
     ablation in Table 3(c)); log2 codes of columns j >= 1 (Eq. 8, which is Eq. 2
     with that s); A_hat = [A[:, 0], s 2^-codes] with column 0 untouched; the
     product A_hat V as the sum of the <start> term and the quantized rest
-    (Eq. 9).  No re-normalisation of A_hat (none is described) and V stays as
-    given (V_hat = V on this path).  Returns O [B, nq, H, d], codes
+    (Eq. 9).  No re-normalisation of A_hat (none is described).  V stays as
+    given (V_hat = V) unless `v_bits` is set, in which case V_hat =
+    `quantize_values(V, v_bits)`.  Returns O [B, nq, H, d], codes
     [B, H, nq, nk-1], s (broadcast shape), A.
     """
     A = softmax_scores(Q, K)
-    V = np.asarray(V, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64) if v_bits is None else quantize_values(V, v_bits)[0]
     if A.shape[-1] < 2:
         raise ValueError("n_k < 2: no score off the <start> column to scale by")
     if fixed_scale is None:

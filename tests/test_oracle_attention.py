@@ -124,3 +124,50 @@ def test_four_bit_agrees_with_eight_bit_below_saturation():
     _, c8, _, _ = oa.cross_attn_logq(Q, K, V, 8)
     _, c4, _, _ = oa.cross_attn_logq(Q, K, V, 4)
     assert np.array_equal(c4[c8 <= 15], c8[c8 <= 15]) and np.all(c4[c8 > 15] == 15)
+
+
+# ---------------------------------------------------------------------------------------------- quantized V_hat
+def test_quantized_values_error_bound_and_grid():
+    """V_hat lies on the grid s (q - Z) of its head's slab and is within s / 2 (+ fp16 rounding) of V."""
+    rng = np.random.default_rng(5)
+    V = rng.normal(0, 1, (2, 9, 3, 8)).astype(np.float16)
+    for bits in (8, 4):
+        V_hat, codes, s, Z = oa.quantize_values(V, bits)
+        assert codes.min() >= 0 and codes.max() <= 2 ** bits - 1
+        span = V.astype(np.float64).max(axis=(1, 3)) - V.astype(np.float64).min(axis=(1, 3))
+        assert np.allclose(s, span / 2 ** bits, rtol=1e-6)                     # Eq. 6 over the slab
+        grid = s[:, None, :, None].astype(np.float64) * (codes - Z[:, None, :, None])
+        assert np.array_equal(V_hat[:, 0], grid[:, 0].astype(np.float32).astype(np.float64))
+        assert np.max(np.abs(V_hat[:, 1:] - grid[:, 1:])) <= 2.0 ** -10 * np.abs(grid).max()   # fp16 operand
+        # interior values round to the nearest level; the top of the range clips by one more half level
+        # (Eq. 6 divides by 2^b, so the maximum maps one level past the last code)
+        err = np.abs(V_hat - V.astype(np.float64))
+        bound = (1.5 * s[:, None, :, None] + 2.0 ** -10 * np.abs(V.astype(np.float64)).max())
+        assert (err <= bound).all()
+        inner = codes < 2 ** bits - 1
+        assert (err[inner] <= (0.5 * s[:, None, :, None] * np.ones_like(err))[inner] * (1 + 1e-6)
+                + 2.0 ** -10 * np.abs(V.astype(np.float64)).max()).all()
+
+
+def test_quantized_values_are_a_fixed_point_on_two_levels():
+    """A slab that holds only its minimum and the value one grid step below its maximum is reproduced."""
+    V = np.zeros((1, 4, 1, 4), np.float16)
+    V[0, 1:, 0, ::2] = 1.0                        # lo = 0, hi = 1 -> s = 2^-8, level 256 clips to 255
+    V_hat, codes, s, Z = oa.quantize_values(V, 8)
+    assert Z[0, 0] == 0 and s[0, 0] == np.float32(2.0 ** -8)
+    assert set(np.unique(codes)) == {0, 255}
+    assert np.array_equal(np.unique(V_hat), np.array([0.0, 255.0 / 256.0]))
+
+
+def test_attention_with_quantized_values_is_eq9_on_v_hat():
+    """cross_attn_logq(v_bits) equals Eq. 9 evaluated with V replaced by quantize_values(V); a wide V_hat
+    grid (16 bits) leaves the output within the grid step of the unquantized-V result."""
+    Q, K, V = synth.attention_inputs(6, 2, 2, 24, 9, 8, ctx_dim=16)
+    O_q, codes, s, A = oa.cross_attn_logq(Q, K, V, 8, v_bits=4)
+    V_hat = oa.quantize_values(V, 4)[0]
+    assert np.array_equal(O_q, oa.split_product(A, codes, s, V_hat))
+    O, _, _, _ = oa.cross_attn_logq(Q, K, V, 8)
+    assert np.max(np.abs(O_q - O)) > 0                                        # 4-bit values do move the output
+    step = oa.quantize_values(V, 4)[2].max()
+    # every output is a combination of values with weights that sum to at most ~1 (+ top-level clip)
+    assert np.max(np.abs(O_q - O)) <= 1.5 * step * 1.01 + 1e-3
