@@ -540,6 +540,7 @@ MICRO_CASES = {
     "conv_8x16x16x1280": ("conv", dict(n=8, h=16, w=16, C=1280, N=1280, G=16)),
     "attn_2x4096x40": ("attn", dict(B=2, H=8, nq=4096, nk=77, d=40)),
     "attn_8x4096x40": ("attn", dict(B=8, H=8, nq=4096, nk=77, d=40)),
+    "attn_qv_2x4096x40": ("attn", dict(B=2, H=8, nq=4096, nk=77, d=40, v_bits=8)),
     "attn_8x1024x80": ("attn", dict(B=8, H=8, nq=1024, nk=77, d=80)),
     "attn_8x256x160": ("attn", dict(B=8, H=8, nq=256, nk=77, d=160)),
 }
@@ -607,7 +608,8 @@ def run_micro(args):
             sets = [(torch.from_numpy(Q).cuda(), torch.from_numpy(K).cuda(), torch.from_numpy(V).cuda(),
                      torch.empty(Q.shape, dtype=torch.float16, device="cuda"),
                      torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")) for _ in range(n_sets)]
-            fns = [lambda s=s: b.cross_attn_logq(s[0], s[1], s[2], 8, out=s[3], workspace=s[4]) for s in sets]
+            fns = [lambda s=s: b.cross_attn_logq(s[0], s[1], s[2], 8, out=s[3], workspace=s[4],
+                                                 v_bits=p.get("v_bits", 0)) for s in sets]
             algo_bytes = 2.0 * Q.size * 2 + 2.0 * K.size * 2
             extra = {}
         reps = max(1, 24 // len(fns))

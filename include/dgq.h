@@ -176,6 +176,17 @@ dgq_status dgq_cross_attn_logq(const void* Q, const void* K, const void* V, int 
                                int d, int score_bits, int scale_gran, const float* fixed_scale, void* O,
                                float* scale_out, uint8_t* codes_out, void* workspace,
                                size_t workspace_bytes, void* stream);
+
+/* The same attention with a quantized value operand V_hat (Eq. 9 writes the product as A_hat V_hat
+ * without naming V's quantizer).  Reading taken here: Eq. 1 with the range of Eq. 6 over one
+ * head's [nk, d] slab of one prompt at `v_bits` (2..8) bits, code decided in fp32,
+ * V_hat = s (q - Z); rows j >= 1 enter the product as fp16, row 0 (<start>) in fp32.  Everything
+ * else, workspace included, as for dgq_cross_attn_logq.  Errors: as there, INVALID_ARG also for
+ * v_bits outside 2..8. */
+dgq_status dgq_cross_attn_logq_qv(const void* Q, const void* K, const void* V, int B, int H, int nq, int nk,
+                                  int d, int score_bits, int scale_gran, const float* fixed_scale, int v_bits,
+                                  void* O, float* scale_out, uint8_t* codes_out, void* workspace,
+                                  size_t workspace_bytes, void* stream);
 dgq_status dgq_cross_attn_workspace_bytes(int B, int H, int nq, int nk, int d, size_t* bytes);
 
 /* ---------------------------------------------------------------- cross-attention without a caller workspace

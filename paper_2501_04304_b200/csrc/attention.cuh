@@ -48,6 +48,7 @@ struct AttnArgs {
   const __half* V;
   __half* O;
   int B, H, nq, nk, d, bits, gran;
+  int v_bits;              // 0: V as given; else V_hat = linear quantizer (Eq. 1, Eq. 6) over the head's [nk, d] slab
   float qk_scale_log2;     // log2(e) / sqrt(d)
   int* smax;               // workspace: ordered-int log2 of the scale per scope
   float2* stats;           // workspace: (row max, log2 row sum) [B][H][nq]
@@ -280,21 +281,68 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_phase2_kernel(const AttnAr
   }
   if (rows_valid > 0) stage_q<D, NKP>(a.Q + (((int64_t)b * a.nq + row0) * a.H + h) * D, q_stride, rows_valid, slab);
   store_k<D, NKP>(xk, sK);
+  // Quantized value operand: range of the head's slab (every CTA of the head derives the same
+  // parameters), codes decided in fp32, de-quantized as s (q - Z); rows j >= 1 become the fp16
+  // operand of the product, row 0 stays fp32.
+  float v_s = 0.f, v_inv = 0.f, v_Zf = 0.f, v_L = 0.f;
+  if (a.v_bits) {
+    __shared__ float v_red[2 * (AT_THREADS / 32)];
+    float lo = INFINITY, hi = -INFINITY;
+#pragma unroll
+    for (int ev = 0; ev < NV; ++ev) {
+      const int i = threadIdx.x + ev * AT_THREADS;
+      if (i / (D / 8) < a.nk) {
+        const __half* xh = reinterpret_cast<const __half*>(&xv[ev]);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float f = __half2float(xh[e]);
+          lo = fminf(lo, f);
+          hi = fmaxf(hi, f);
+        }
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+      hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    if (lane == 0) {
+      v_red[warp] = lo;
+      v_red[AT_THREADS / 32 + warp] = hi;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < AT_THREADS / 32; ++w) {
+      lo = fminf(lo, v_red[w]);
+      hi = fmaxf(hi, v_red[AT_THREADS / 32 + w]);
+    }
+    int v_Z;
+    group_params(lo, hi, a.v_bits, v_s, v_inv, v_Z);
+    v_Zf = (float)v_Z;
+    v_L = (float)((1 << a.v_bits) - 1);
+  }
 #pragma unroll
   for (int ev = 0; ev < NV; ++ev) {
     const int i = threadIdx.x + ev * AT_THREADS;
     if (i >= NKP * 16 * (D / 8)) continue;
     const int j = i / (D / 8), v = i - j * (D / 8);
     const __half* xh = reinterpret_cast<const __half*>(&xv[ev]);
+    float f[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      f[e] = __half2float(xh[e]);
+      if (a.v_bits && j < a.nk)
+        f[e] = __fmul_rn(v_s, __fsub_rn((float)quantize_code(f[e], v_inv, v_Zf, v_L), v_Zf));
+    }
     if (j == 0) {
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
-        sV0[v * 8 + e] = __half2float(xh[e]);
+        sV0[v * 8 + e] = f[e];
         sVt[(v * 8 + e) * Cfg::LDV] = __float2half(0.f);
       }
     } else {
 #pragma unroll
-      for (int e = 0; e < 8; ++e) sVt[(v * 8 + e) * Cfg::LDV + j] = xh[e];
+      for (int e = 0; e < 8; ++e) sVt[(v * 8 + e) * Cfg::LDV + j] = __float2half_rn(f[e]);
     }
   }
   __syncthreads();
@@ -433,12 +481,13 @@ extern "C" dgq_status dgq_cross_attn_workspace_bytes(int B, int H, int nq, int n
   return DGQ_OK;
 }
 
-extern "C" dgq_status dgq_cross_attn_logq(const void* Q, const void* K, const void* V, int B, int H, int nq, int nk,
-                                          int d, int score_bits, int scale_gran, const float* fixed_scale, void* O,
-                                          float* scale_out, uint8_t* codes_out, void* workspace,
-                                          size_t workspace_bytes, void* stream) {
-  using namespace dgq;
+namespace dgq {
+static dgq_status attn_run(const void* Q, const void* K, const void* V, int B, int H, int nq, int nk, int d,
+                           int score_bits, int scale_gran, const float* fixed_scale, int v_bits, void* O,
+                           float* scale_out, uint8_t* codes_out, void* workspace, size_t workspace_bytes,
+                           void* stream) {
   if (!Q || !K || !V || !O || B <= 0 || H <= 0 || nq <= 0 || d <= 0) return DGQ_ERR_INVALID_ARG;
+  if (v_bits != 0 && (v_bits < 2 || v_bits > 8)) return DGQ_ERR_INVALID_ARG;
   if (nk < 2) return DGQ_ERR_INVALID_ARG;
   if (score_bits < 2 || score_bits > 8) return DGQ_ERR_INVALID_ARG;
   if (scale_gran < DGQ_SCALE_PER_PROMPT || scale_gran > DGQ_SCALE_PER_CALL) return DGQ_ERR_INVALID_ARG;
@@ -460,6 +509,7 @@ extern "C" dgq_status dgq_cross_attn_logq(const void* Q, const void* K, const vo
   a.d = d;
   a.bits = score_bits;
   a.gran = scale_gran;
+  a.v_bits = v_bits;
   a.qk_scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)d));
   a.smax = (int*)workspace;
   a.stats = (float2*)((char*)workspace + attn_smax_bytes(B, H));
@@ -477,4 +527,22 @@ extern "C" dgq_status dgq_cross_attn_logq(const void* Q, const void* K, const vo
     case 128: return launch_attn_d<128>(a, st);
     default: return launch_attn_d<160>(a, st);
   }
+}
+}  // namespace dgq
+
+extern "C" dgq_status dgq_cross_attn_logq(const void* Q, const void* K, const void* V, int B, int H, int nq, int nk,
+                                          int d, int score_bits, int scale_gran, const float* fixed_scale, void* O,
+                                          float* scale_out, uint8_t* codes_out, void* workspace,
+                                          size_t workspace_bytes, void* stream) {
+  return dgq::attn_run(Q, K, V, B, H, nq, nk, d, score_bits, scale_gran, fixed_scale, 0, O, scale_out, codes_out,
+                       workspace, workspace_bytes, stream);
+}
+
+extern "C" dgq_status dgq_cross_attn_logq_qv(const void* Q, const void* K, const void* V, int B, int H, int nq,
+                                             int nk, int d, int score_bits, int scale_gran, const float* fixed_scale,
+                                             int v_bits, void* O, float* scale_out, uint8_t* codes_out,
+                                             void* workspace, size_t workspace_bytes, void* stream) {
+  if (v_bits < 2 || v_bits > 8) return DGQ_ERR_INVALID_ARG;
+  return dgq::attn_run(Q, K, V, B, H, nq, nk, d, score_bits, scale_gran, fixed_scale, v_bits, O, scale_out,
+                       codes_out, workspace, workspace_bytes, stream);
 }

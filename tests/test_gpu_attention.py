@@ -9,11 +9,13 @@ from dgq_testlib import gpu, to_dev, check_output
 pytestmark = pytest.mark.gpu
 
 
-def _compare(torch, b, Q, K, V, bits, gran=0, fixed=None, code_frac=1e-4, out_rel=1e-3):
-    O_ref, codes_ref, s_ref, A = oa.cross_attn_logq(Q, K, V, bits, gran, fixed)
+def _compare(torch, b, Q, K, V, bits, gran=0, fixed=None, code_frac=1e-4, out_rel=1e-3, v_bits=None):
+    O_ref, codes_ref, s_ref, A = oa.cross_attn_logq(Q, K, V, bits, gran, fixed, v_bits=v_bits)
     fx = to_dev(torch, np.asarray(fixed, np.float32)) if fixed is not None else None
     O, scale, codes = b.cross_attn_logq(to_dev(torch, Q), to_dev(torch, K), to_dev(torch, V), bits, gran, fx,
-                                        want_scale=True, want_codes=True)
+                                        want_scale=True, want_codes=True, v_bits=v_bits or 0)
+    if v_bits:
+        V = oa.quantize_values(V, v_bits)[0]      # the value operand both sides multiply with
     assert b.device_status() == 0
     s_gpu = scale.cpu().numpy().astype(np.float64)
     assert np.allclose(s_gpu, s_ref.ravel(), rtol=2e-5, atol=0)
@@ -88,3 +90,27 @@ def test_argument_errors():
     with pytest.raises(b.DgqError) as e:
         b.cross_attn_logq(Qd, Kd, Vd, workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
     assert e.value.status == 4
+
+
+@pytest.mark.parametrize("v_bits", [8, 6, 4])
+def test_quantized_value_operand(v_bits):
+    """Eq. 9 with V_hat: the kernel quantizes each head's value slab itself; the oracle's V_hat enters the
+    comparison, so a wrong range, zero-point or code shows as an output error far above the tolerance."""
+    torch, b = gpu()
+    Q, K, V = synth.attention_inputs(8, 2, 4, 300, 77, 40)
+    _compare(torch, b, Q, K, V, 8, v_bits=v_bits)
+
+
+@pytest.mark.parametrize("B,H,nq,nk,d", [(1, 2, 64, 77, 160), (2, 2, 40, 128, 128), (3, 1, 129, 2, 40), (1, 3, 257, 100, 64)])
+def test_quantized_value_operand_shapes(B, H, nq, nk, d):
+    torch, b = gpu()
+    Q, K, V = synth.attention_inputs(9, B, H, nq, nk, d, ctx_dim=64)
+    _compare(torch, b, Q, K, V, 8, code_frac=5e-4, v_bits=8)
+
+
+def test_quantized_value_operand_rejects_bad_bits():
+    torch, b = gpu()
+    Q, K, V = [to_dev(torch, x) for x in synth.attention_inputs(10, 1, 1, 16, 4, 40, ctx_dim=16)]
+    for bad in (1, 9):
+        with pytest.raises(Exception):
+            b.cross_attn_logq(Q, K, V, 8, v_bits=bad)
