@@ -101,3 +101,31 @@ def attention_reference(Q, K, V):
     """Plain softmax attention softmax(Q K^T / sqrt(d)) V in fp64 (no quantization)."""
     A = softmax_scores(Q, K)
     return np.einsum("bhqk,bkhd->bqhd", A, np.asarray(V, dtype=np.float64))
+
+
+def self_attn_logq(Q, K, V, bits, fixed_scale=None):
+    """Log2-quantized attention scores without a <start> column (self-attention, Sec. 3.3: the log
+    quantizer of Eq. 2 is applied "to both self and cross-attentions"), fp64 throughout.
+
+    A = softmax(Q K^T / sqrt(d)) (Eq. 3); codes = clamp(rint(-log2(A / s)), 0, 2^b - 1) over ALL keys
+    (Eq. 2); A_hat = s 2^-codes; O = A_hat V.  The paper gives the dynamic scale only for
+    cross-attention; reading (parity unpinned): s is the largest score of each query row unless
+    `fixed_scale` ([B], one per prompt) is given.  No re-normalisation, V as given.
+    Q [B, nq, H, d], K, V [B, nk, H, d] -> O [B, nq, H, d], codes [B, H, nq, nk], s (broadcast shape), A.
+    """
+    A = softmax_scores(Q, K)
+    V = np.asarray(V, dtype=np.float64)
+    if fixed_scale is None:
+        s = np.maximum(A.max(axis=-1, keepdims=True), FLT_MIN)
+    else:
+        s = np.maximum(np.asarray(fixed_scale, dtype=np.float64).reshape(-1, 1, 1, 1), FLT_MIN)
+    s_full = np.broadcast_to(s, A.shape[:-1] + (1,))
+    codes = log_quantize(A, s_full, bits)
+    return self_product(codes, s, V), codes, s, A
+
+
+def self_product(codes, s, V):
+    """O = (s 2^-codes) V for given codes [B, H, nq, nk], fp64."""
+    V = np.asarray(V, dtype=np.float64)
+    s_full = np.broadcast_to(s, codes.shape[:-1] + (1,))
+    return np.einsum("bhqk,bkhd->bqhd", log_dequantize(codes, s_full), V)

@@ -171,3 +171,48 @@ def test_attention_with_quantized_values_is_eq9_on_v_hat():
     step = oa.quantize_values(V, 4)[2].max()
     # every output is a combination of values with weights that sum to at most ~1 (+ top-level clip)
     assert np.max(np.abs(O_q - O)) <= 1.5 * step * 1.01 + 1e-3
+
+
+# ---------------------------------------------------------------------------------------------- self-attention
+def test_self_attention_uniform_scores_are_exact():
+    """Q = 0: every score is 1 / n_k, the row maximum is the scale, every code is 0 and the output is the
+    plain mean of V, exactly what unquantized attention gives."""
+    rng = np.random.default_rng(11)
+    B, nq, nk, H, d = 2, 5, 7, 3, 4
+    Q = np.zeros((B, nq, H, d), np.float16)
+    K = rng.normal(0, 1, (B, nk, H, d)).astype(np.float16)
+    V = rng.normal(0, 1, (B, nk, H, d)).astype(np.float16)
+    O, codes, s, A = oa.self_attn_logq(Q, K, V, 8)
+    assert not codes.any()
+    assert np.allclose(s, 1.0 / nk)
+    assert np.allclose(O, np.broadcast_to(V.astype(np.float64).mean(axis=1)[:, None], O.shape), atol=1e-12)
+    assert np.allclose(O, oa.attention_reference(Q, K, V), atol=1e-12)
+
+
+def test_self_attention_log_levels_and_error_bound():
+    """Eq. 2 with the row maximum as scale: the largest score of a row gets code 0 and is reproduced; every
+    unclamped score is reproduced within a factor 2^(+-1/2); codes grow by one per halving of the score."""
+    Q, K, V = synth.attention_inputs(12, 2, 2, 20, 33, 8, ctx_dim=16)
+    O, codes, s, A = oa.self_attn_logq(Q, K, V, 8)
+    imax = A.argmax(axis=-1)
+    assert (np.take_along_axis(codes, imax[..., None], axis=-1) == 0).all()
+    A_hat = s * np.exp2(-codes.astype(np.float64))
+    assert np.allclose(np.take_along_axis(A_hat, imax[..., None], axis=-1), A.max(axis=-1, keepdims=True))
+    free = codes < 255
+    ratio = A_hat[free] / A[free]
+    assert ratio.min() >= 2.0 ** -0.5 - 1e-12 and ratio.max() <= 2.0 ** 0.5 + 1e-12
+    assert np.array_equal(codes, np.clip(np.rint(-np.log2(A / s)), 0, 255).astype(np.int64))
+    assert np.array_equal(O, oa.self_product(codes, s, V))
+
+
+def test_self_attention_fixed_scale_and_clamping():
+    """A fixed scale of 1 (the largest value a softmax score can take) with 3 bits: scores below 2^-7.5 all
+    take the last code; the output is the explicit sum over keys."""
+    Q, K, V = synth.attention_inputs(13, 1, 1, 6, 40, 8, ctx_dim=16)
+    O, codes, s, A = oa.self_attn_logq(Q, K, V, 3, fixed_scale=np.array([1.0]))
+    assert codes.max() == 7 and (codes[A < 2.0 ** -7.5] == 7).all()
+    want = np.zeros_like(O)
+    for q in range(6):
+        for k in range(40):
+            want[0, q, 0] += 2.0 ** -int(codes[0, 0, q, k]) * V[0, k, 0].astype(np.float64)
+    assert np.allclose(O, want, atol=1e-12)
