@@ -187,6 +187,18 @@ dgq_status dgq_cross_attn_logq_qv(const void* Q, const void* K, const void* V, i
                                   int d, int score_bits, int scale_gran, const float* fixed_scale, int v_bits,
                                   void* O, float* scale_out, uint8_t* codes_out, void* workspace,
                                   size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------- self-attention (Eq. 2, Eq. 3; Sec. 3.3
+ * applies the log quantizer "to both self and cross-attentions")
+ * Q dev fp16 [B, nq, H, d]; K, V dev fp16 [B, nk, H, d]; O dev fp16 [B, nq, H, d]; any nk >= 1.
+ * A = softmax(Q K^T / sqrt(d)) in fp32; codes = clamp(rint(-log2(A / s)), 0, 2^bits - 1) over ALL keys
+ * (there is no <start> column here); O = s * sum_j 2^-code_j V[j].  s is the largest score of each query
+ * row, or fixed_scale[b] (dev [B]) when non-NULL; the paper states the dynamic scale for cross-attention
+ * only, the row maximum is this library's reading.  codes_out (dev u8 [B, H, nq, nk]) is optional.
+ * No workspace: the keys are walked twice by the same thread block.  d in {40, 64, 80, 128, 160}.
+ * Errors: INVALID_ARG, ALIGNMENT, UNSUPPORTED, CUDA. */
+dgq_status dgq_self_attn_logq(const void* Q, const void* K, const void* V, int B, int H, int nq, int nk, int d,
+                              int score_bits, const float* fixed_scale, void* O, uint8_t* codes_out, void* stream);
 dgq_status dgq_cross_attn_workspace_bytes(int B, int H, int nq, int nk, int d, size_t* bytes);
 
 /* ---------------------------------------------------------------- cross-attention without a caller workspace

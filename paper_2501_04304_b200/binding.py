@@ -26,7 +26,7 @@ SCALE_PER_PROMPT, SCALE_PER_PROMPT_HEAD, SCALE_PER_CALL = 0, 1, 2
 EXPORTS = [
     "dgq_calibrate_groups", "dgq_groups_from_host", "dgq_groups_destroy", "dgq_groups_info",
     "dgq_groups_export", "dgq_quantize_act", "dgq_weight_prepare", "dgq_weight_from_codes",
-    "dgq_weight_destroy", "dgq_weight_export", "dgq_linear", "dgq_cross_attn_logq", "dgq_cross_attn_logq_qv",
+    "dgq_weight_destroy", "dgq_weight_export", "dgq_linear", "dgq_cross_attn_logq", "dgq_cross_attn_logq_qv", "dgq_self_attn_logq",
     "dgq_cross_attn_workspace_bytes", "dgq_cross_attn_logq_noalloc", "dgq_device_status", "dgq_status_string", "dgq_launch_count",
 ]
 
@@ -282,6 +282,20 @@ def cross_attn_logq(Q, K, V, score_bits=8, scale_gran=SCALE_PER_PROMPT, fixed_sc
                                    _ptr(scale), _ptr(codes), _ptr(ws), C.c_size_t(ws.numel()), _stream(stream))
     _check(st, "dgq_cross_attn_logq")
     return O, scale, codes
+
+
+def self_attn_logq(Q, K, V, score_bits=8, fixed_scale=None, out=None, want_codes=False, stream=None):
+    """dgq_self_attn_logq.  Q [B, nq, H, d], K, V [B, nk, H, d] CUDA fp16.  Returns (O, codes)."""
+    B, nq, H, d = Q.shape
+    nk = K.shape[1]
+    assert Q.is_contiguous() and K.is_contiguous() and V.is_contiguous()
+    O = out if out is not None else torch.empty_like(Q)
+    codes = torch.empty((B, H, nq, nk), dtype=torch.uint8, device=Q.device) if want_codes else None
+    st = lib().dgq_self_attn_logq(_ptr(Q), _ptr(K), _ptr(V), C.c_int(B), C.c_int(H), C.c_int(nq), C.c_int(nk),
+                                  C.c_int(d), C.c_int(score_bits), _ptr(fixed_scale), _ptr(O), _ptr(codes),
+                                  _stream(stream))
+    _check(st, "dgq_self_attn_logq")
+    return O, codes
 
 
 NOALLOC_MAX_ROWS = 1 << 18
