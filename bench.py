@@ -543,6 +543,9 @@ MICRO_CASES = {
     "attn_qv_2x4096x40": ("attn", dict(B=2, H=8, nq=4096, nk=77, d=40, v_bits=8)),
     "attn_8x1024x80": ("attn", dict(B=8, H=8, nq=1024, nk=77, d=80)),
     "attn_8x256x160": ("attn", dict(B=8, H=8, nq=256, nk=77, d=160)),
+    "selfattn_2x4096x40": ("selfattn", dict(B=2, H=8, n=4096, d=40)),
+    "selfattn_8x1024x80": ("selfattn", dict(B=8, H=8, n=1024, d=80)),
+    "selfattn_8x256x160": ("selfattn", dict(B=8, H=8, n=256, d=160)),
 }
 
 
@@ -599,6 +602,16 @@ def run_micro(args):
                 algo_ops = 2.0 * M * p["N"] * kreal
                 algo_bytes = M * C + p["N"] * kreal * wb / 8 + 2.0 * M * p["N"]
             extra = {"K_pad": g.K_pad, "G": g.G}
+        elif kind == "selfattn":
+            rng = np.random.default_rng(SEED)
+            shape = (p["B"], p["n"], p["H"], p["d"])
+            n_sets = max(2, int(3 * 126e6 // (4 * 2 * np.prod(shape))) + 1)
+            sets = [tuple(torch.from_numpy(rng.normal(0, 1, shape).astype(np.float16)).cuda() for _ in range(3))
+                    + (torch.empty(shape, dtype=torch.float16, device="cuda"),) for _ in range(n_sets)]
+            fns = [lambda s=s: b.self_attn_logq(s[0], s[1], s[2], 8, out=s[3]) for s in sets]
+            algo_bytes = 4.0 * 2 * np.prod(shape)
+            algo_ops = 4.0 * p["B"] * p["H"] * p["n"] * p["n"] * p["d"]      # Q K^T and P V, once each
+            extra = {}
         else:
             a = p
             Q, K, V = synth.attention_inputs(SEED, a["B"], a["H"], a["nq"], a["nk"], a["d"])
@@ -638,7 +651,10 @@ def run_micro(args):
                "sets": len(fns), **extra}
         if algo_ops:
             rec["tops"] = algo_ops / us / 1e6
-            rec["frac_int8_peak"] = rec["tops"] / (2 * peaks["bf16"])
+            if kind == "selfattn":      # fp16 operands: the measured bf16 peak is the denominator
+                rec["frac_f16_peak"] = rec["tops"] / peaks["bf16"]
+            else:
+                rec["frac_int8_peak"] = rec["tops"] / (2 * peaks["bf16"])
         assert b.device_status() == 0
         print(json.dumps(rec), flush=True)
         del sets, fns, graph

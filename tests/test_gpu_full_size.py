@@ -8,6 +8,7 @@ from oracle import linear as ol
 from paper_2501_04304_b200 import synth
 from dgq_testlib import gpu, to_dev, unpermute_codes
 from test_gpu_attention import _compare
+from oracle import attention as oa
 
 pytestmark = pytest.mark.gpu
 
@@ -90,6 +91,28 @@ def test_attention_full_size():
     torch, b = gpu()
     Q, K, V = synth.attention_inputs(23, 2, 8, 4096, 77, 40)
     _compare(torch, b, Q, K, V, 8)
+
+
+def test_self_attention_full_size_sampled_rows():
+    """4096 tokens attending to 4096 keys (the 64 x 64 level): every query row is independent with a per-row
+    scale, so the oracle computes sampled rows against all keys and those rows are compared in full."""
+    torch, b = gpu()
+    B, H, n, d = 2, 8, 4096, 40
+    rng = np.random.default_rng(41)
+    Q = rng.normal(0, 1, (B, n, H, d)).astype(np.float16)
+    K = rng.normal(0, 1, (B, n, H, d)).astype(np.float16)
+    V = rng.normal(0, 1, (B, n, H, d)).astype(np.float16)
+    O, codes = b.self_attn_logq(to_dev(torch, Q), to_dev(torch, K), to_dev(torch, V), 8, want_codes=True)
+    torch.cuda.synchronize()
+    assert b.device_status() == 0
+    rows = _sample_rows(n, 5)[::2]
+    O_ref, codes_ref, s_ref, _ = oa.self_attn_logq(Q[:, rows], K, V, 8)
+    c = codes[:, :, torch.from_numpy(rows).cuda()].cpu().numpy().astype(np.int64)
+    diff = np.abs(c - codes_ref)
+    assert diff.max() <= 1 and (diff != 0).mean() <= 3e-4
+    O_alt = oa.self_product(c, s_ref, V)
+    Og = O[:, torch.from_numpy(rows).cuda()].float().cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(Og - O_alt)) <= REL * np.max(np.abs(O_alt))
 
 
 def test_chained_layers_in_a_graph_match_serialised_calls():
