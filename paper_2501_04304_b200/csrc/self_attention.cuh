@@ -315,34 +315,3 @@ static dgq_status launch_self_attn(const SelfAttnArgs& a, cudaStream_t stream) {
 
 }  // namespace dgq
 
-extern "C" dgq_status dgq_self_attn_logq(const void* Q, const void* K, const void* V, int B, int H, int nq, int nk,
-                                         int d, int score_bits, const float* fixed_scale, void* O,
-                                         uint8_t* codes_out, void* stream) {
-  using namespace dgq;
-  if (!Q || !K || !V || !O || B <= 0 || H <= 0 || nq <= 0 || nk <= 0 || d <= 0) return DGQ_ERR_INVALID_ARG;
-  if (score_bits < 2 || score_bits > 8) return DGQ_ERR_INVALID_ARG;
-  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return DGQ_ERR_ALIGNMENT;
-  if (d != 40 && d != 64 && d != 80 && d != 128 && d != 160) return DGQ_ERR_UNSUPPORTED;
-  SelfAttnArgs a;
-  a.Q = (const __half*)Q;
-  a.K = (const __half*)K;
-  a.V = (const __half*)V;
-  a.O = (__half*)O;
-  a.B = B;
-  a.H = H;
-  a.nq = nq;
-  a.nk = nk;
-  a.bits = score_bits;
-  a.qk_scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)d));
-  a.fixed_scale = fixed_scale;
-  a.codes_out = codes_out;
-  a.n_row_blocks = 0;
-  cudaStream_t st = (cudaStream_t)stream;
-  switch (d) {
-    case 40: return launch_self_attn<40>(a, st);
-    case 64: return launch_self_attn<64>(a, st);
-    case 80: return launch_self_attn<80>(a, st);
-    case 128: return launch_self_attn<128>(a, st);
-    default: return launch_self_attn<160>(a, st);
-  }
-}
