@@ -9,7 +9,7 @@
 #include "weights.cuh"
 #include "linear.cuh"
 #include "attention.cuh"
-#include "self_attention_tc.cuh"
+#include "self_attention.cuh"
 
 // ---------------------------------------------------------------------------------------------
 // Cross-attention for callers that cannot allocate a workspace: the scratch is this fixed array

@@ -1,24 +1,28 @@
-// Attention with log2-quantized softmax scores and no <start> column (self-attention; Sec. 3.3
-// applies the log quantizer of Eq. 2 "to both self and cross-attentions"):
-//     A = softmax(Q K^T / sqrt(d)),  code = clamp(rint(-log2(A / s)), 0, 2^b - 1),  O = s sum_j 2^-code_j V_j
-// with s the largest score of the query row, or one fixed scale per prompt.
+// Self-attention with log2-quantized scores (Sec. 3.3 applies the log quantizer of Eq. 2 "to both self
+// and cross-attentions") on the tcgen05 tensor cores:
 //
-// The key axis is as long as the query axis (up to 4096), so the keys are walked in blocks of 64
-// twice by the same CTA: the first walk keeps a running maximum and sum of every row (the softmax
-// statistics), the second recomputes the logits, forms the codes in the log domain and multiplies
-// with the block of V.  No workspace and no second kernel: with a per-row or fixed scale nothing has
-// to be reduced across CTAs.  One CTA = one (prompt, head, block of query rows); K and V^T blocks
-// are loaded into registers one block ahead and parked in shared memory between two CTA barriers.
-// The building blocks (shared-memory layouts, warp-level MMA fragments, the fp16 exponent-field
-// construction of 2^-code) are those of the cross-attention kernels.
+//     A = softmax(Q K^T / sqrt(d)),  code = clamp(rint(-log2(A / s)), 0, 2^b - 1),  O = s sum_j 2^-code_j V_j
+//
+// with s the largest score of the query row, or one fixed scale per prompt; there is no <start> column.
+// One CTA owns one or two tiles of 128 query rows of one (prompt, head) and walks the keys in blocks of
+// 128 two or three times:
+//   walk "max"   : S = Q K^T into tensor memory, every row keeps its largest logit;
+//   walk "sum"   : (fixed scale only) the row sums of 2^(t - max), which the codes then depend on;
+//   walk "codes" : S again; code = rint(base - t) in the log domain, P = 2^(14 - code) as fp16 into a
+//                  shared-memory operand tile, O += P V on the tensor cores.  With the row maximum as
+//                  scale the codes do not depend on the row sum, which is then gathered in this walk.
+// Roles: 16 softmax warps (warp w reads tensor-memory lanes 32 (w % 4) .. +31, columns 32 (w / 4) .. +31
+// of every score tile), one TMA producer lane, one MMA issuer lane.  With two query tiles the softmax
+// warps alternate between them, so every K / V block fetched from L2 serves 256 query rows and one
+// tile's MMAs run under the other tile's arithmetic.  Q, K and P are K-major operands with 128-byte
+// swizzled rows; V is used as it lies in memory (features contiguous), an MN-major operand.  Tiles are
+// fetched as boxes of 64 features x 128 tokens; features beyond d and tokens beyond the sequence are
+// zero-filled by the copy engine, so d = 40 runs as 48 and ragged ends need no staging.
 #pragma once
 
 #include "attention.cuh"
 
 namespace dgq {
-
-constexpr int SA_NKP = 4;            // 16-key pairs per block
-constexpr int SA_KB = SA_NKP * 16;   // keys per block
 
 struct SelfAttnArgs {
   const __half* Q;
@@ -32,286 +36,508 @@ struct SelfAttnArgs {
   int n_row_blocks;
 };
 
-// 64 keys of K starting at key0 (rows and features beyond the real ones zero) into registers / smem.
-template <int D>
-__device__ __forceinline__ void sa_load_k(const SelfAttnArgs& a, int b, int h, int key0,
-                                          uint4 (&x)[KStage<D, SA_NKP>::N]) {
-  constexpr int VEC = KStage<D, SA_NKP>::VEC;
-#pragma unroll
-  for (int e = 0; e < KStage<D, SA_NKP>::N; ++e) {
-    const int i = threadIdx.x + e * AT_THREADS;
-    const int j = i / VEC, v = i - j * VEC;
-    x[e] = make_uint4(0, 0, 0, 0);
-    if (i < SA_KB * VEC && key0 + j < a.nk && v < D / 8)
-      x[e] = __ldg(reinterpret_cast<const uint4*>(a.K + (((int64_t)b * a.nk + key0 + j) * a.H + h) * D) + v);
-  }
-}
+constexpr int SATC_SOFTMAX_WARPS = 16;
+constexpr int SATC_WARP_TMA = 16;
+constexpr int SATC_WARP_MMA = 17;
+constexpr int SATC_THREADS = 18 * 32;
+constexpr int SATC_BQ = 128;            // query rows per tile
+constexpr int SATC_BK = 128;            // keys per block
+constexpr int SATC_PANEL = 128 * 128;   // bytes of one 64-feature (or 64-key) panel of 128 rows
+constexpr int SATC_TMEM_O = 256;        // first column of the output accumulators (score buffers at 0 and 128)
 
 template <int D>
-struct SaVStage {
-  static constexpr int N = (SA_KB * (D / 8) + AT_THREADS - 1) / AT_THREADS;
+struct SaTcCfg {
+  static constexpr int DP = (D + 15) / 16 * 16;
+  static constexpr int NP = (D + 63) / 64;
+  static constexpr int NT = NP == 1 ? 2 : 1;   // query tiles per CTA (shared memory and tensor memory budget)
+  static constexpr int KSTEPS = DP / 16;
+  static constexpr int KST = NP == 1 ? 3 : (NP == 2 ? 2 : 1);
+  static constexpr int VST = NP == 1 ? 2 : 1;
+  static constexpr int PST = NP <= 2 ? 2 : 1;
+  static constexpr int TILE = NP * SATC_PANEL;
+  static constexpr int P_TILE = 2 * SATC_PANEL;
+  static constexpr int OFF_K = NT * TILE;
+  static constexpr int OFF_V = OFF_K + KST * TILE;
+  static constexpr int OFF_P = OFF_V + VST * TILE;
+  static constexpr int OFF_SH = OFF_P + PST * P_TILE;
+  static constexpr int SMEM = 1024 + OFF_SH + 1024 + 2 * 4 * SATC_BQ * 4;
+  static_assert(SMEM <= 232448, "shared memory budget");
+  static_assert(SATC_TMEM_O + NT * DP <= 512, "tensor memory budget");
 };
-template <int D>
-__device__ __forceinline__ void sa_load_v(const SelfAttnArgs& a, int b, int h, int key0, uint4 (&x)[SaVStage<D>::N]) {
-#pragma unroll
-  for (int e = 0; e < SaVStage<D>::N; ++e) {
-    const int i = threadIdx.x + e * AT_THREADS;
-    const int j = i / (D / 8), v = i - j * (D / 8);
-    x[e] = make_uint4(0, 0, 0, 0);
-    if (i < SA_KB * (D / 8) && key0 + j < a.nk)
-      x[e] = __ldg(reinterpret_cast<const uint4*>(a.V + (((int64_t)b * a.nk + key0 + j) * a.H + h) * D) + v);
-  }
+
+struct SaTcShared {
+  uint64_t q_full;
+  uint64_t k_full[3], k_empty[3];
+  uint64_t v_full[2], v_empty[2];
+  uint64_t s_full[2], s_free[2];
+  uint64_t p_full[2], p_free[2];
+  uint64_t o_full;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                        uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
 }
-// V block written transposed: sVt[feature][key in block]; keys beyond nk hold zeros.
-template <int D>
-__device__ __forceinline__ void sa_store_vt(const uint4 (&x)[SaVStage<D>::N], __half* sVt) {
-  constexpr int LDV = AttnCfg<D, SA_NKP>::LDV;
-#pragma unroll
-  for (int e = 0; e < SaVStage<D>::N; ++e) {
-    const int i = threadIdx.x + e * AT_THREADS;
-    if (i >= SA_KB * (D / 8)) continue;
-    const int j = i / (D / 8), v = i - j * (D / 8);
-    const __half* xh = reinterpret_cast<const __half*>(&x[e]);
-#pragma unroll
-    for (int q = 0; q < 8; ++q) sVt[(v * 8 + q) * LDV + j] = xh[q];
-  }
+// MN-major operand with 128-byte swizzled rows (one row = 64 contiguous elements of the M/N axis for
+// one k): `lbo` = bytes between 64-element blocks of the M/N axis, `sbo` = bytes between groups of 8 k.
+__device__ __forceinline__ uint64_t smem_desc_mn(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ void named_bar_sync(int id, int n_threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
 }
 
-// Base-2 logits of the warp's rows against the 64 keys in shared memory; keys >= keys_left get -inf.
-template <int D>
-__device__ __forceinline__ void sa_logits(const __half* slab, const __half* sK, int keys_left, float qk_scale_log2,
-                                          float (&S)[AttnCfg<D, SA_NKP>::MT][2 * SA_NKP][4]) {
-  using Cfg = AttnCfg<D, SA_NKP>;
-  const int lane = threadIdx.x & 31;
-  const int r = lane >> 2, c = lane & 3;
-#pragma unroll
-  for (int mt = 0; mt < Cfg::MT; ++mt)
-#pragma unroll
-    for (int nt = 0; nt < Cfg::NT; ++nt)
-#pragma unroll
-      for (int i = 0; i < 4; ++i) S[mt][nt][i] = 0.f;
-#pragma unroll
-  for (int kk = 0; kk < Cfg::KS; ++kk) {
-    uint32_t af[Cfg::MT][4];
-#pragma unroll
-    for (int mt = 0; mt < Cfg::MT; ++mt)
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-        af[mt][i] = *reinterpret_cast<const uint32_t*>(slab + (mt * 16 + r + (i & 1) * 8) * Cfg::LDK + kk * 16 +
-                                                       2 * c + (i >> 1) * 8);
-#pragma unroll
-    for (int nt = 0; nt < Cfg::NT; ++nt) {
-      const __half* kp = sK + (nt * 8 + r) * Cfg::LDK + kk * 16 + 2 * c;
-      const uint32_t b0 = *reinterpret_cast<const uint32_t*>(kp);
-      const uint32_t b1 = *reinterpret_cast<const uint32_t*>(kp + 8);
-#pragma unroll
-      for (int mt = 0; mt < Cfg::MT; ++mt) mma_f16(S[mt][nt], af[mt][0], af[mt][1], af[mt][2], af[mt][3], b0, b1);
-    }
-  }
-#pragma unroll
-  for (int mt = 0; mt < Cfg::MT; ++mt)
-#pragma unroll
-    for (int nt = 0; nt < Cfg::NT; ++nt)
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int key = nt * 8 + 2 * c + (i & 1);
-        S[mt][nt][i] = key < keys_left ? S[mt][nt][i] * qk_scale_log2 : -INFINITY;
-      }
+// kind::f16 instruction descriptor: fp32 accumulator (bits 4-5 = 1), fp16 A and B (format 0), B major at
+// bit 16 (1 = MN-major), N >> 3 at bit 17, M >> 4 at bit 24.
+__host__ __device__ constexpr uint32_t satc_idesc(int n, bool b_mn_major) {
+  return (1u << 4) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(SATC_BQ >> 4) << 24);
 }
 
-template <int D, bool CODES>
-__global__ void __launch_bounds__(AT_THREADS, 1) self_attn_logq_kernel(const SelfAttnArgs a) {
-  using Cfg = AttnCfg<D, SA_NKP>;
-  constexpr int NT_O = D / 8;
-  extern __shared__ __align__(16) unsigned char at_smem[];
-  __half* sK = reinterpret_cast<__half*>(at_smem);
-  __half* sQ = reinterpret_cast<__half*>(at_smem + Cfg::SM_K);
-  __half* sVt = reinterpret_cast<__half*>(at_smem + Cfg::SM_K + Cfg::SM_Q);  // [D][LDV]
+
+template <int D, bool FIXED, bool CODES>
+__global__ void __launch_bounds__(SATC_THREADS, 1)
+self_attn_logq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                      const __grid_constant__ CUtensorMap tmV, const __grid_constant__ SelfAttnArgs a) {
+  using Cfg = SaTcCfg<D>;
+  constexpr int NP = Cfg::NP, NT = Cfg::NT, KST = Cfg::KST, VST = Cfg::VST, PST = Cfg::PST;
+  constexpr int N_WALKS = FIXED ? 3 : 2;
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) &
+                                                         ~uintptr_t(1023));
+  unsigned char* sQ = smem;
+  unsigned char* sK = smem + Cfg::OFF_K;
+  unsigned char* sV = smem + Cfg::OFF_V;
+  unsigned char* sP = smem + Cfg::OFF_P;
+  SaTcShared* sh = reinterpret_cast<SaTcShared*>(smem + Cfg::OFF_SH);
+  float* mpart = reinterpret_cast<float*>(smem + Cfg::OFF_SH + 1024);  // [4][128] partial row maxima
+  float* zpart = mpart + 4 * SATC_BQ;                                  // [4][128] partial row sums
+  volatile int* abort_flag = &sh->abort_flag;
+
   const int blk = blockIdx.x;
   const int rb = blk % a.n_row_blocks;
   const int h = (blk / a.n_row_blocks) % a.H;
   const int b = blk / (a.n_row_blocks * a.H);
+  const int row0 = rb * (SATC_BQ * NT);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int r = lane >> 2, c = lane & 3;
-  const int row0 = rb * Cfg::ROWS + warp * Cfg::WROWS;
-  const int rows_valid = min(Cfg::WROWS, a.nq - row0);  // may be <= 0: the warp still helps with the loads
-  const int64_t q_stride = (int64_t)a.H * D;
-  __half* slab = sQ + warp * Cfg::WROWS * Cfg::LDK;
-  const int n_blocks = (a.nk + SA_KB - 1) / SA_KB;
+  const int nb = (a.nk + SATC_BK - 1) / SATC_BK;
+  const int per_walk = nb * NT;  // score tiles per walk, in the order (key block, query tile)
+
   pdl_launch_dependents();
+  if (threadIdx.x == 0) {
+    mbar_init(&sh->q_full, 1);
+    for (int i = 0; i < 3; ++i) {
+      mbar_init(&sh->k_full[i], 1);
+      mbar_init(&sh->k_empty[i], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&sh->v_full[i], 1);
+      mbar_init(&sh->v_empty[i], 1);
+      mbar_init(&sh->s_full[i], 1);
+      mbar_init(&sh->s_free[i], SATC_SOFTMAX_WARPS);
+      mbar_init(&sh->p_full[i], SATC_SOFTMAX_WARPS);
+      mbar_init(&sh->p_free[i], 1);
+    }
+    mbar_init(&sh->o_full, 1);
+    sh->abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == SATC_WARP_MMA) {
+    tmem_alloc(&sh->tmem_base, 512);
+    tmem_relinquish();
+  }
   pdl_wait();  // Q, K and V may come from earlier kernels
-  uint4 xk[KStage<D, SA_NKP>::N];
-  sa_load_k<D>(a, b, h, 0, xk);
-  if (rows_valid > 0) stage_q<D, SA_NKP>(a.Q + (((int64_t)b * a.nq + row0) * a.H + h) * D, q_stride, rows_valid, slab);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = sh->tmem_base;
 
-  // ---- first walk over the keys: running maximum and sum of 2^(t - max) of every row
-  float m[Cfg::MT][2], z[Cfg::MT][2];
-#pragma unroll
-  for (int mt = 0; mt < Cfg::MT; ++mt)
-#pragma unroll
-    for (int hi = 0; hi < 2; ++hi) {
-      m[mt][hi] = -INFINITY;
-      z[mt][hi] = 0.f;
-    }
-  for (int kb = 0; kb < n_blocks; ++kb) {
-    __syncthreads();  // everyone is done with the previous block
-    store_k<D, SA_NKP>(xk, sK);
-    __syncthreads();
-    if (kb + 1 < n_blocks) sa_load_k<D>(a, b, h, (kb + 1) * SA_KB, xk);  // travels during the arithmetic
-    if (rows_valid > 0) {
-      float S[Cfg::MT][Cfg::NT][4];
-      sa_logits<D>(slab, sK, a.nk - kb * SA_KB, a.qk_scale_log2, S);
-#pragma unroll
-      for (int mt = 0; mt < Cfg::MT; ++mt)
-#pragma unroll
-        for (int hi = 0; hi < 2; ++hi) {
-          float tmax = -INFINITY;
-#pragma unroll
-          for (int nt = 0; nt < Cfg::NT; ++nt)
-#pragma unroll
-            for (int i = 0; i < 2; ++i) tmax = fmaxf(tmax, S[mt][nt][hi * 2 + i]);
-          tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
-          tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
-          const float mn = fmaxf(m[mt][hi], tmax);  // finite: every block holds at least one real key
-          float zz = 0.f;
-#pragma unroll
-          for (int nt = 0; nt < Cfg::NT; ++nt)
-#pragma unroll
-            for (int i = 0; i < 2; ++i) zz += ex2_approx(S[mt][nt][hi * 2 + i] - mn);
-          zz += __shfl_xor_sync(0xffffffffu, zz, 1);
-          zz += __shfl_xor_sync(0xffffffffu, zz, 2);
-          z[mt][hi] = z[mt][hi] * ex2_approx(m[mt][hi] - mn) + zz;
-          m[mt][hi] = mn;
+  if (warp == SATC_WARP_TMA) {
+    // ------------------------------------------------------------ TMA producer (one lane)
+    if (lane == 0) {
+      tma_prefetch_desc(&tmQ);
+      tma_prefetch_desc(&tmK);
+      tma_prefetch_desc(&tmV);
+      mbar_arrive_expect_tx(&sh->q_full, (uint32_t)(NT * Cfg::TILE));
+      for (int t = 0; t < NT; ++t)
+        for (int p = 0; p < NP; ++p)
+          tma_load_4d(sQ + t * Cfg::TILE + p * SATC_PANEL, &tmQ, &sh->q_full, p * 64, h, row0 + t * SATC_BQ, b);
+      uint32_t kit = 0, vit = 0;
+      auto load_v = [&](int j) {
+        const uint32_t vs = vit % VST;
+        mbar_wait_lean(smem_u32(&sh->v_empty[vs]), ((vit / VST) & 1u) ^ 1u, abort_flag);
+        mbar_arrive_expect_tx(&sh->v_full[vs], (uint32_t)Cfg::TILE);
+        for (int p = 0; p < NP; ++p)
+          tma_load_4d(sV + vs * Cfg::TILE + p * SATC_PANEL, &tmV, &sh->v_full[vs], p * 64, h, j * SATC_BK, b);
+        ++vit;
+      };
+      for (int w = 0; w < N_WALKS && !*abort_flag; ++w) {
+        const bool last = (w == N_WALKS - 1);
+        for (int j = 0; j < nb; ++j) {
+          const uint32_t ks = kit % KST;
+          mbar_wait_lean(smem_u32(&sh->k_empty[ks]), ((kit / KST) & 1u) ^ 1u, abort_flag);
+          mbar_arrive_expect_tx(&sh->k_full[ks], (uint32_t)Cfg::TILE);
+          for (int p = 0; p < NP; ++p)
+            tma_load_4d(sK + ks * Cfg::TILE + p * SATC_PANEL, &tmK, &sh->k_full[ks], p * 64, h, j * SATC_BK, b);
+          ++kit;
+          // V of the previous block goes out after K of this one: the scores of block j are issued
+          // before P V of block j - 1, and a V stage only frees when such a product has completed
+          if (last && j > 0) load_v(j - 1);
+          if (*abort_flag) break;
         }
-    }
-  }
-  // code = rint(base - t) with base = log2 s + max + log2 sum; with the row maximum as scale
-  // (s = 1 / sum) this is the row maximum of the logits itself
-  float base[Cfg::MT][2], s_out[Cfg::MT][2];
-  {
-    const float log2_fixed = a.fixed_scale ? log2f(fmaxf(__ldg(a.fixed_scale + b), 1.17549435e-38f)) : 0.f;
-#pragma unroll
-    for (int mt = 0; mt < Cfg::MT; ++mt)
-#pragma unroll
-      for (int hi = 0; hi < 2; ++hi) {
-        const float lz = log2f(z[mt][hi]);
-        const float log2s = a.fixed_scale ? log2_fixed : -lz;
-        base[mt][hi] = a.fixed_scale ? log2_fixed + m[mt][hi] + lz : m[mt][hi];
-        s_out[mt][hi] = exp2f(log2s - AT_P_SHIFT);
+        if (last && !*abort_flag) load_v(nb - 1);
       }
-  }
-
-  // ---- second walk: codes and the product with V
-  const float Lf = (float)((1 << a.bits) - 1);
-  const float Lcap = fminf(Lf, AT_CODE_CAP);
-  float acc[Cfg::MT][NT_O][4];
-#pragma unroll
-  for (int mt = 0; mt < Cfg::MT; ++mt)
-#pragma unroll
-    for (int nt = 0; nt < NT_O; ++nt)
-#pragma unroll
-      for (int i = 0; i < 4; ++i) acc[mt][nt][i] = 0.f;
-  uint4 xv[SaVStage<D>::N];
-  sa_load_k<D>(a, b, h, 0, xk);
-  sa_load_v<D>(a, b, h, 0, xv);
-  for (int kb = 0; kb < n_blocks; ++kb) {
-    __syncthreads();
-    store_k<D, SA_NKP>(xk, sK);
-    sa_store_vt<D>(xv, sVt);
-    __syncthreads();
-    if (kb + 1 < n_blocks) {
-      sa_load_k<D>(a, b, h, (kb + 1) * SA_KB, xk);
-      sa_load_v<D>(a, b, h, (kb + 1) * SA_KB, xv);
     }
-    if (rows_valid > 0) {
-      float S[Cfg::MT][Cfg::NT][4];
-      sa_logits<D>(slab, sK, a.nk - kb * SA_KB, a.qk_scale_log2, S);
-      uint32_t pa[Cfg::MT][SA_NKP][4];  // A fragments of A_hat / s * 2^14
+    __syncwarp();
+  } else if (warp == SATC_WARP_MMA) {
+    // ------------------------------------------------------------ MMA issuer (one lane)
+    // Score tiles are numbered g = 0 .. N_WALKS * per_walk - 1.  S(g + 1) is issued as soon as its
+    // buffer has been read (early in the arithmetic of tile g - 1) and before P V of tile g - 1, whose
+    // P tile only completes when that arithmetic ends: the tensor pipe is never what a softmax warp
+    // waits for.
+    if (lane == 0) {
+      constexpr uint32_t IDESC_QK = satc_idesc(SATC_BK, false);
+      constexpr uint32_t IDESC_PV = satc_idesc(Cfg::DP, true);
+      const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV), p_addr = smem_u32(sP);
+      const int total = N_WALKS * per_walk;
+      uint32_t kit = 0, vit = 0;
+      auto issue_qk = [&](int g) {
+        const int t = g % NT;
+        const uint32_t ks = kit % KST, sb = (uint32_t)g & 1u;
+        if (t == 0) mbar_wait_lean(smem_u32(&sh->k_full[ks]), (kit / KST) & 1u, abort_flag);
+        mbar_wait_lean(smem_u32(&sh->s_free[sb]), (((uint32_t)g >> 1) & 1u) ^ 1u, abort_flag);
+        tc_fence_after();
 #pragma unroll
-      for (int mt = 0; mt < Cfg::MT; ++mt)
+        for (int kstep = 0; kstep < Cfg::KSTEPS; ++kstep) {
+          const uint32_t off = (kstep >> 2) * SATC_PANEL + (kstep & 3) * 32;
+          mma_f16(tmem_base + sb * SATC_BK, smem_desc(q_addr + t * Cfg::TILE + off, 1024, 2),
+                  smem_desc(k_addr + ks * Cfg::TILE + off, 1024, 2), IDESC_QK, kstep > 0 ? 1u : 0u);
+        }
+        if (t == NT - 1) {
+          mma_commit(&sh->k_empty[ks]);
+          ++kit;
+        }
+        mma_commit(&sh->s_full[sb]);
+      };
+      // O(tile) += P V for codes-walk tile number c (= key block c / NT, query tile c % NT)
+      auto issue_pv = [&](int c) {
+        const int t = c % NT, jj = c / NT;
+        const uint32_t pb = (uint32_t)c % PST, vs = vit % VST;
+        mbar_wait_lean(smem_u32(&sh->p_full[pb]), ((uint32_t)c / PST) & 1u, abort_flag);
+        if (t == 0) mbar_wait_lean(smem_u32(&sh->v_full[vs]), (vit / VST) & 1u, abort_flag);
+        tc_fence_after();
 #pragma unroll
-        for (int hi = 0; hi < 2; ++hi) {
+        for (int kstep = 0; kstep < SATC_BK / 16; ++kstep) {
+          const uint64_t da = smem_desc(p_addr + pb * Cfg::P_TILE + (kstep >> 2) * SATC_PANEL + (kstep & 3) * 32, 1024, 2);
+          const uint64_t db = smem_desc_mn(v_addr + vs * Cfg::TILE + kstep * 2048, SATC_PANEL, 1024);
+          mma_f16(tmem_base + SATC_TMEM_O + t * Cfg::DP, da, db, IDESC_PV, (jj > 0 || kstep > 0) ? 1u : 0u);
+        }
+        if (t == NT - 1) {
+          mma_commit(&sh->v_empty[vs]);
+          ++vit;
+        }
+        mma_commit(&sh->p_free[pb]);
+      };
+      mbar_wait_lean(smem_u32(&sh->q_full), 0, abort_flag);
+      const int first_code = (N_WALKS - 1) * per_walk;
+      issue_qk(0);
+      for (int g = 0; g < total && !*abort_flag; ++g) {
+        if (g + 1 < total) issue_qk(g + 1);
+        if (g - 1 >= first_code) issue_pv(g - 1 - first_code);
+      }
+      if (!*abort_flag) {
+        issue_pv(per_walk - 1);
+        mma_commit(&sh->o_full);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------ softmax / quantizer warps
+    const int q = warp & 3, cp = warp >> 2;
+    const int row = q * 32 + lane;  // row of a query tile
+    const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
+    const float scale = a.qk_scale_log2;
+    const unsigned long long nscale2 = pack_f32x2(-scale, -scale);
+    const unsigned long long one2 = pack_f32x2(1.f, 1.f);
+    const unsigned long long magic2 = pack_f32x2(12582912.0f, 12582912.0f);
+    const uint32_t L = (1u << a.bits) - 1u;
+    const uint32_t code_top = 0x4B400000u + L;                                 // bits of 1.5 * 2^23 + last code
+    const uint32_t p_top = 0x4B400000u + min(L, (uint32_t)AT_CODE_CAP);       // ... + last code with a non-zero fp16 weight
+    float m_raw[NT], m2[NT], base[NT];
+    unsigned long long zsum2[NT];
 #pragma unroll
-          for (int nt = 0; nt < Cfg::NT; ++nt) {
-            float p[2];
+    for (int t = 0; t < NT; ++t) {
+      m_raw[t] = -INFINITY;
+      m2[t] = 0.f;
+      base[t] = 0.f;
+      zsum2[t] = 0ull;
+    }
+    uint32_t g = 0, c = 0;  // score tiles / codes-walk tiles seen so far
+    for (int w = 0; w < N_WALKS; ++w) {
+      const bool walk_max = (w == 0), walk_codes = (w == N_WALKS - 1);
+      for (int j = 0; j < nb; ++j) {
+        const int valid = a.nk - j * SATC_BK - cp * 32;  // this warp's columns below `valid` are real keys
 #pragma unroll
-            for (int i = 0; i < 2; ++i) {
-              const float t = S[mt][nt][hi * 2 + i];
-              // rint by adding 1.5 * 2^23: the low bits of the sum are the integer.  -inf logits
-              // (keys beyond nk) clamp to the cap; their V^T columns are zero.
-              const float x = fminf(fmaxf(base[mt][hi] - t, 0.f), CODES ? Lf : Lcap);
-              const int code = __float_as_int(x + 12582912.0f) - 0x4B400000;
-              if (CODES) {
-                const int key = kb * SA_KB + nt * 8 + 2 * c + i;
-                const int orow = mt * 16 + r + hi * 8;
-                if (key < a.nk && orow < rows_valid)
-                  a.codes_out[(((int64_t)b * a.H + h) * a.nq + row0 + orow) * a.nk + key] = (uint8_t)code;
-              }
-              p[i] = __int_as_float((127 + (int)AT_P_SHIFT - min(code, (int)AT_CODE_CAP)) << 23);
+        for (int t = 0; t < NT; ++t) {
+          const uint32_t sb = g & 1u;
+          // After a time-out every wait returns at once and the loops run to their ends on whatever the
+          // buffers hold (an error is recorded): no warp leaves early, so the named barriers below are
+          // always reached by all 16 warps.
+          mbar_wait_lean(smem_u32(&sh->s_full[sb]), (g >> 1) & 1u, abort_flag);
+          __syncwarp();
+          tc_fence_after();
+          uint32_t r[32];
+          {
+            uint32_t r0[16], r1[16];
+            tmem_ld16(t_lane + sb * SATC_BK + cp * 32, r0);
+            tmem_ld16(t_lane + sb * SATC_BK + cp * 32 + 16, r1);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              r[i] = r0[i];
+              r[16 + i] = r1[i];
             }
-            const __half2 ph = __floats2half2_rn(p[0], p[1]);
-            pa[mt][nt >> 1][(nt & 1) * 2 + hi] = *reinterpret_cast<const uint32_t*>(&ph);
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sh->s_free[sb]);
+          ++g;
+          if (valid < 32) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (i >= valid) r[i] = 0xFF800000u;  // -inf
+          }
+          if (walk_max) {
+            float mx0 = m_raw[t], mx1 = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+              mx0 = fmaxf(mx0, __uint_as_float(r[i]));
+              mx1 = fmaxf(mx1, __uint_as_float(r[i + 1]));
+            }
+            m_raw[t] = fmaxf(mx0, mx1);
+          } else if (!walk_codes) {
+            // row sums with the final maximum (fixed scale: the codes need them first)
+            float z0 = 0.f, z1 = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+              z0 += ex2_approx(fmaf(__uint_as_float(r[i]), scale, -m2[t]));
+              z1 += ex2_approx(fmaf(__uint_as_float(r[i + 1]), scale, -m2[t]));
+            }
+            zsum2[t] = pack_f32x2(__uint_as_float((uint32_t)zsum2[t]) + z0, __uint_as_float((uint32_t)(zsum2[t] >> 32)) + z1);
+          } else {
+            const uint32_t pb = c % PST;
+            const int64_t code_row =
+                (((int64_t)b * a.H + h) * a.nq + row0 + t * SATC_BQ + row) * a.nk + j * SATC_BK + cp * 32;
+            const unsigned long long base2 = pack_f32x2(base[t], base[t]);
+            unsigned char* prow = sP + pb * Cfg::P_TILE + (cp >> 1) * SATC_PANEL + row * 128;
+            unsigned long long zs = zsum2[t];
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4) {
+              uint32_t pk[4];
+#pragma unroll
+              for (int i2 = 0; i2 < 4; ++i2) {
+                const int i = c4 * 8 + i2 * 2;
+                // x = base - t * scale >= 0 up to rounding (the row maximum has code 0); -inf logits (keys
+                // beyond nk) give +inf, which the integer minimum below clamps to the last code
+                unsigned long long x2 = fma_f32x2(pack_f32x2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), nscale2, base2);
+                float x0, x1;
+                unpack_f32x2(x2, x0, x1);
+                if (!FIXED) {
+                  // 2^(t - max) = 2^-x for the row sum
+                  zs = fma_f32x2(pack_f32x2(ex2_approx(-x0), ex2_approx(-x1)), one2, zs);
+                } else {
+                  x2 = pack_f32x2(fmaxf(x0, 0.f), fmaxf(x1, 0.f));  // a fixed scale can lie below a score
+                }
+                // rint by adding 1.5 * 2^23: the low bits of the sum are the integer
+                float y0, y1;
+                unpack_f32x2(fma_f32x2(x2, one2, magic2), y0, y1);
+                const uint32_t b0 = __float_as_uint(y0), b1 = __float_as_uint(y1);
+                if (CODES) {
+                  r[i] = min(b0, code_top) & 0xFFu;
+                  r[i + 1] = min(b1, code_top) & 0xFFu;
+                }
+                // 2^(14 - code) as fp32 bits: (127 + 14) << 23 minus code << 23 (the bits of 1.5 * 2^23 shift out)
+                const float p0 = __uint_as_float(0x46800000u - (min(b0, p_top) << 23));
+                const float p1 = __uint_as_float(0x46800000u - (min(b1, p_top) << 23));
+                const __half2 ph = __floats2half2_rn(p0, p1);
+                pk[i2] = *reinterpret_cast<const uint32_t*>(&ph);
+              }
+              if (c4 == 0) {
+                mbar_wait_lean(smem_u32(&sh->p_free[pb]), ((c / PST) & 1u) ^ 1u, abort_flag);
+                __syncwarp();
+              }
+              *reinterpret_cast<uint4*>(prow + ((((cp & 1) * 4 + c4) ^ (row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            }
+            zsum2[t] = zs;
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh->p_full[pb]);
+            ++c;
+            if (CODES && row0 + t * SATC_BQ + row < a.nq) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (i < valid) a.codes_out[code_row + i] = (uint8_t)r[i];
+            }
           }
         }
+      }
+      if (walk_max) {
 #pragma unroll
-      for (int kk = 0; kk < SA_NKP; ++kk)
-#pragma unroll
-        for (int nt = 0; nt < NT_O; ++nt) {
-          const __half* vp = sVt + (nt * 8 + r) * Cfg::LDV + kk * 16 + 2 * c;
-          const uint32_t b0 = *reinterpret_cast<const uint32_t*>(vp);
-          const uint32_t b1 = *reinterpret_cast<const uint32_t*>(vp + 8);
-#pragma unroll
-          for (int mt = 0; mt < Cfg::MT; ++mt)
-            mma_f16(acc[mt][nt], pa[mt][kk][0], pa[mt][kk][1], pa[mt][kk][2], pa[mt][kk][3], b0, b1);
+        for (int t = 0; t < NT; ++t) {
+          if (t > 0) named_bar_sync(1, SATC_SOFTMAX_WARPS * 32);  // the exchange buffer is read out
+          mpart[cp * SATC_BQ + row] = m_raw[t];
+          named_bar_sync(1, SATC_SOFTMAX_WARPS * 32);
+          m_raw[t] = fmaxf(fmaxf(mpart[row], mpart[SATC_BQ + row]), fmaxf(mpart[2 * SATC_BQ + row], mpart[3 * SATC_BQ + row]));
+          m2[t] = m_raw[t] * scale;
+          base[t] = m2[t];  // row maximum as scale: log2 s + max + log2 sum = max
         }
+      } else if (!walk_codes) {
+        const float log2_fixed = log2f(fmaxf(__ldg(a.fixed_scale + b), 1.17549435e-38f));
+#pragma unroll
+        for (int t = 0; t < NT; ++t) {
+          if (t > 0) named_bar_sync(1, SATC_SOFTMAX_WARPS * 32);
+          zpart[cp * SATC_BQ + row] = __uint_as_float((uint32_t)zsum2[t]) + __uint_as_float((uint32_t)(zsum2[t] >> 32));
+          named_bar_sync(1, SATC_SOFTMAX_WARPS * 32);
+          const float z = (zpart[row] + zpart[SATC_BQ + row]) + (zpart[2 * SATC_BQ + row] + zpart[3 * SATC_BQ + row]);
+          base[t] = log2_fixed + m2[t] + log2f(z);
+        }
+      }
+    }
+    float s_row[NT];
+#pragma unroll
+    for (int t = 0; t < NT; ++t) {
+      if (FIXED) {
+        s_row[t] = fmaxf(__ldg(a.fixed_scale + b), 1.17549435e-38f);
+      } else {
+        if (t > 0) named_bar_sync(1, SATC_SOFTMAX_WARPS * 32);
+        zpart[cp * SATC_BQ + row] = __uint_as_float((uint32_t)zsum2[t]) + __uint_as_float((uint32_t)(zsum2[t] >> 32));
+        named_bar_sync(1, SATC_SOFTMAX_WARPS * 32);
+        s_row[t] = 1.0f / ((zpart[row] + zpart[SATC_BQ + row]) + (zpart[2 * SATC_BQ + row] + zpart[3 * SATC_BQ + row]));
+      }
+      s_row[t] *= 6.103515625e-05f;  // 2^-14
+    }
+    mbar_wait_lean(smem_u32(&sh->o_full), 0, abort_flag);
+    __syncwarp();
+    tc_fence_after();
+#pragma unroll
+    for (int t = 0; t < NT; ++t) {
+      const int orow = row0 + t * SATC_BQ + row;
+      __half* o_row = a.O + (((int64_t)b * a.nq + orow) * a.H + h) * D;
+      for (int ch = cp; ch < D / 8; ch += 4) {
+        uint32_t o[8];
+        tmem_ld8(t_lane + SATC_TMEM_O + t * Cfg::DP + ch * 8, o);
+        tmem_ld_wait();
+        __half2 oh[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          oh[i] = __floats2half2_rn(s_row[t] * __uint_as_float(o[2 * i]), s_row[t] * __uint_as_float(o[2 * i + 1]));
+        if (orow < a.nq) *(reinterpret_cast<uint4*>(o_row) + ch) = *reinterpret_cast<const uint4*>(oh);
+      }
     }
   }
-  if (rows_valid <= 0) return;
-  // O = s 2^-14 acc, staged in the warp's slab (its Q rows are no longer needed) and written with 128-bit stores
-  __syncwarp();
-#pragma unroll
-  for (int nt = 0; nt < NT_O; ++nt) {
-    const int col = nt * 8 + 2 * c;
-#pragma unroll
-    for (int mt = 0; mt < Cfg::MT; ++mt)
-#pragma unroll
-      for (int hi = 0; hi < 2; ++hi)
-        *reinterpret_cast<__half2*>(slab + (mt * 16 + r + hi * 8) * Cfg::LDK + col) =
-            __floats2half2_rn(s_out[mt][hi] * acc[mt][nt][hi * 2], s_out[mt][hi] * acc[mt][nt][hi * 2 + 1]);
+
+  // ------------------------------------------------------------ common exit
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    // give copies that may still be in flight time to land before the CTA's shared memory is released
+    const long long t0 = clock64();
+    while (clock64() - t0 < 200000) {
+    }
+    __syncthreads();
   }
-  __syncwarp();
-  __half* o_base = a.O + (((int64_t)b * a.nq + row0) * a.H + h) * D;
-  for (int i = lane; i < Cfg::WROWS * (D / 8); i += 32) {
-    const int rr = i / (D / 8), v = i - rr * (D / 8);
-    if (rr < rows_valid)
-      *(reinterpret_cast<uint4*>(o_base + rr * q_stride) + v) = *reinterpret_cast<const uint4*>(slab + rr * Cfg::LDK + v * 8);
+  if (warp == SATC_WARP_MMA) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
   }
 }
 
-template <int D>
-static dgq_status launch_self_attn(const SelfAttnArgs& a, cudaStream_t stream) {
-  using Cfg = AttnCfg<D, SA_NKP>;
-  constexpr int SM = Cfg::SMEM2;
+// [B, n, H, d] fp16 as a 4-D tensor (d, H, n, B); boxes of 64 features x 128 tokens of one head.
+static bool satc_encode(CUtensorMap* m, const void* base, int B, int n, int H, int d) {
+  const uint64_t dims[4] = {(uint64_t)d, (uint64_t)H, (uint64_t)n, (uint64_t)B};
+  const uint64_t strides[3] = {(uint64_t)d * 2, (uint64_t)H * d * 2, (uint64_t)n * H * d * 2};
+  const uint32_t box[4] = {64, 1, 128, 1};
+  return encode_map(m, base, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_DATA_TYPE_FLOAT16);
+}
+
+template <int D, bool FIXED, bool CODES>
+static dgq_status launch_self_attn2(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
+                                       const SelfAttnArgs& a, unsigned grid, cudaStream_t stream) {
+  using Cfg = SaTcCfg<D>;
   static bool attr_set[64] = {false};
   int dev = 0;
   DGQ_CUDA_OK(cudaGetDevice(&dev));
   if (dev >= 64 || !attr_set[dev]) {
-    DGQ_CUDA_OK(cudaFuncSetAttribute(self_attn_logq_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM));
-    DGQ_CUDA_OK(cudaFuncSetAttribute(self_attn_logq_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM));
+    DGQ_CUDA_OK(cudaFuncSetAttribute(self_attn_logq_kernel<D, FIXED, CODES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     Cfg::SMEM));
     if (dev < 64) attr_set[dev] = true;
   }
-  SelfAttnArgs aa = a;
-  aa.n_row_blocks = (a.nq + Cfg::ROWS - 1) / Cfg::ROWS;
-  const int64_t grid = (int64_t)a.B * a.H * aa.n_row_blocks;
-  if (grid > INT_MAX) return DGQ_ERR_UNSUPPORTED;
-  if (a.codes_out)
-    DGQ_CUDA_OK(launch_pdl(self_attn_logq_kernel<D, true>, dim3((unsigned)grid), dim3(AT_THREADS), (size_t)SM, stream, aa));
-  else
-    DGQ_CUDA_OK(launch_pdl(self_attn_logq_kernel<D, false>, dim3((unsigned)grid), dim3(AT_THREADS), (size_t)SM, stream, aa));
+  DGQ_CUDA_OK(launch_pdl(self_attn_logq_kernel<D, FIXED, CODES>, dim3(grid), dim3(SATC_THREADS), (size_t)Cfg::SMEM, stream,
+                         tmQ, tmK, tmV, a));
   g_launches += 1;
   DGQ_CUDA_OK(cudaGetLastError());
   return DGQ_OK;
 }
 
+template <int D>
+static dgq_status launch_self_attn(const SelfAttnArgs& a, cudaStream_t stream) {
+  SelfAttnArgs aa = a;
+  aa.n_row_blocks = (a.nq + SATC_BQ * SaTcCfg<D>::NT - 1) / (SATC_BQ * SaTcCfg<D>::NT);
+  const int64_t grid = (int64_t)a.B * a.H * aa.n_row_blocks;
+  if (grid > INT_MAX) return DGQ_ERR_UNSUPPORTED;
+  CUtensorMap tmQ, tmK, tmV;
+  std::memset(&tmQ, 0, sizeof(tmQ));
+  std::memset(&tmK, 0, sizeof(tmK));
+  std::memset(&tmV, 0, sizeof(tmV));
+  if (!satc_encode(&tmQ, a.Q, a.B, a.nq, a.H, D) || !satc_encode(&tmK, a.K, a.B, a.nk, a.H, D) ||
+      !satc_encode(&tmV, a.V, a.B, a.nk, a.H, D))
+    return DGQ_ERR_CUDA;
+  const unsigned g = (unsigned)grid;
+  if (a.fixed_scale)
+    return a.codes_out ? launch_self_attn2<D, true, true>(tmQ, tmK, tmV, aa, g, stream)
+                       : launch_self_attn2<D, true, false>(tmQ, tmK, tmV, aa, g, stream);
+  return a.codes_out ? launch_self_attn2<D, false, true>(tmQ, tmK, tmV, aa, g, stream)
+                     : launch_self_attn2<D, false, false>(tmQ, tmK, tmV, aa, g, stream);
+}
+
 }  // namespace dgq
 
+extern "C" dgq_status dgq_self_attn_logq(const void* Q, const void* K, const void* V, int B, int H, int nq, int nk,
+                                         int d, int score_bits, const float* fixed_scale, void* O,
+                                         uint8_t* codes_out, void* stream) {
+  using namespace dgq;
+  if (!Q || !K || !V || !O || B <= 0 || H <= 0 || nq <= 0 || nk <= 0 || d <= 0) return DGQ_ERR_INVALID_ARG;
+  if (score_bits < 2 || score_bits > 8) return DGQ_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return DGQ_ERR_ALIGNMENT;
+  if (d != 40 && d != 64 && d != 80 && d != 128 && d != 160) return DGQ_ERR_UNSUPPORTED;
+  SelfAttnArgs a;
+  a.Q = (const __half*)Q;
+  a.K = (const __half*)K;
+  a.V = (const __half*)V;
+  a.O = (__half*)O;
+  a.B = B;
+  a.H = H;
+  a.nq = nq;
+  a.nk = nk;
+  a.bits = score_bits;
+  a.qk_scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)d));
+  a.fixed_scale = fixed_scale;
+  a.codes_out = codes_out;
+  a.n_row_blocks = 0;
+  cudaStream_t st = (cudaStream_t)stream;
+  switch (d) {
+    case 40: return launch_self_attn<40>(a, st);
+    case 64: return launch_self_attn<64>(a, st);
+    case 80: return launch_self_attn<80>(a, st);
+    case 128: return launch_self_attn<128>(a, st);
+    default: return launch_self_attn<160>(a, st);
+  }
+}
