@@ -12,7 +12,8 @@
 //                  shared-memory operand tile, O += P V on the tensor cores.  With the row maximum as
 //                  scale the codes do not depend on the row sum, which is then gathered in this walk.
 // Roles: 16 softmax warps (warp w reads tensor-memory lanes 32 (w % 4) .. +31, columns 32 (w / 4) .. +31
-// of every score tile), one TMA producer lane, one MMA issuer lane.  With two query tiles the softmax
+// of every score tile), one TMA producer lane, one lane that issues the score MMAs and one that issues
+// the P V MMAs (each tile costs an issuing thread a chain of dependent instructions, so the two run apart).  With two query tiles the softmax
 // warps alternate between them, so every K / V block fetched from L2 serves 256 query rows and one
 // tile's MMAs run under the other tile's arithmetic.  Q, K and P are K-major operands with 128-byte
 // swizzled rows; V is used as it lies in memory (features contiguous), an MN-major operand.  Tiles are
@@ -38,8 +39,9 @@ struct SelfAttnArgs {
 
 constexpr int SATC_SOFTMAX_WARPS = 16;
 constexpr int SATC_WARP_TMA = 16;
-constexpr int SATC_WARP_MMA = 17;
-constexpr int SATC_THREADS = 18 * 32;
+constexpr int SATC_WARP_MMA = 17;   // issues S = Q K^T (and owns the tensor-memory allocation)
+constexpr int SATC_WARP_PV = 18;    // issues O += P V
+constexpr int SATC_THREADS = 19 * 32;
 constexpr int SATC_BQ = 128;            // query rows per tile
 constexpr int SATC_BK = 128;            // keys per block
 constexpr int SATC_PANEL = 128 * 128;   // bytes of one 64-feature (or 64-key) panel of 128 rows
@@ -83,6 +85,20 @@ __device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t desc_a, uint64
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// The same with the descriptors given as (low, high) words: the high words are constants of the layout,
+// only the address field in the low word changes from step to step, which keeps the issuing thread's
+// dependent instruction chain short (that chain, not the tensor pipe, is what bounds a tile otherwise).
+__device__ __forceinline__ void mma_f16_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
+                                             uint32_t b_hi, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %2};\n\t"
+      "mov.b64 db, {%3, %4};\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 // MN-major operand with 128-byte swizzled rows (one row = 64 contiguous elements of the M/N axis for
@@ -197,65 +213,81 @@ self_attn_logq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     }
     __syncwarp();
   } else if (warp == SATC_WARP_MMA) {
-    // ------------------------------------------------------------ MMA issuer (one lane)
-    // Score tiles are numbered g = 0 .. N_WALKS * per_walk - 1.  S(g + 1) is issued as soon as its
-    // buffer has been read (early in the arithmetic of tile g - 1) and before P V of tile g - 1, whose
-    // P tile only completes when that arithmetic ends: the tensor pipe is never what a softmax warp
-    // waits for.
+    // ------------------------------------------------------------ score issuer (one lane)
+    // Score tiles are numbered g = 0 .. N_WALKS * per_walk - 1 in the order (walk, key block, query
+    // tile) and alternate between the two score buffers; a tile is issued as soon as its buffer has
+    // been read, which is early in the arithmetic of tile g - 2.
     if (lane == 0) {
       constexpr uint32_t IDESC_QK = satc_idesc(SATC_BK, false);
-      constexpr uint32_t IDESC_PV = satc_idesc(Cfg::DP, true);
-      const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV), p_addr = smem_u32(sP);
+      constexpr uint32_t HI = smem_desc_hi(1024, 2);
+      const uint32_t q_lo = smem_desc_lo(smem_u32(sQ)), k_lo = smem_desc_lo(smem_u32(sK));
+      const uint32_t k_full0 = smem_u32(&sh->k_full[0]), k_empty0 = smem_u32(&sh->k_empty[0]);
+      const uint32_t s_full0 = smem_u32(&sh->s_full[0]), s_free0 = smem_u32(&sh->s_free[0]);
       const int total = N_WALKS * per_walk;
-      uint32_t kit = 0, vit = 0;
-      auto issue_qk = [&](int g) {
-        const int t = g % NT;
-        const uint32_t ks = kit % KST, sb = (uint32_t)g & 1u;
-        if (t == 0) mbar_wait_lean(smem_u32(&sh->k_full[ks]), (kit / KST) & 1u, abort_flag);
-        mbar_wait_lean(smem_u32(&sh->s_free[sb]), (((uint32_t)g >> 1) & 1u) ^ 1u, abort_flag);
+      uint32_t ks = 0, k_par = 0;
+      mbar_wait_lean(smem_u32(&sh->q_full), 0, abort_flag);
+      for (int g = 0; g < total; ++g) {
+        const uint32_t sb = (uint32_t)g & 1u;
+        const uint32_t t = NT == 2 ? sb : 0u;
+        if (t == 0) mbar_wait_lean(k_full0 + ks * 8u, k_par, abort_flag);
+        mbar_wait_lean(s_free0 + sb * 8u, (((uint32_t)g >> 1) & 1u) ^ 1u, abort_flag);
         tc_fence_after();
+        const uint32_t a_lo = q_lo + t * (uint32_t)(Cfg::TILE >> 4), b_lo = k_lo + ks * (uint32_t)(Cfg::TILE >> 4);
 #pragma unroll
         for (int kstep = 0; kstep < Cfg::KSTEPS; ++kstep) {
-          const uint32_t off = (kstep >> 2) * SATC_PANEL + (kstep & 3) * 32;
-          mma_f16(tmem_base + sb * SATC_BK, smem_desc(q_addr + t * Cfg::TILE + off, 1024, 2),
-                  smem_desc(k_addr + ks * Cfg::TILE + off, 1024, 2), IDESC_QK, kstep > 0 ? 1u : 0u);
+          const uint32_t off = (uint32_t)(((kstep >> 2) * SATC_PANEL + (kstep & 3) * 32) >> 4);
+          mma_f16_lohi(tmem_base + sb * SATC_BK, a_lo + off, HI, b_lo + off, HI, IDESC_QK, kstep > 0 ? 1u : 0u);
         }
         if (t == NT - 1) {
-          mma_commit(&sh->k_empty[ks]);
-          ++kit;
+          mma_commit_addr(k_empty0 + ks * 8u);
+          if (++ks == (uint32_t)KST) {
+            ks = 0;
+            k_par ^= 1u;
+          }
         }
-        mma_commit(&sh->s_full[sb]);
-      };
-      // O(tile) += P V for codes-walk tile number c (= key block c / NT, query tile c % NT)
-      auto issue_pv = [&](int c) {
-        const int t = c % NT, jj = c / NT;
-        const uint32_t pb = (uint32_t)c % PST, vs = vit % VST;
-        mbar_wait_lean(smem_u32(&sh->p_full[pb]), ((uint32_t)c / PST) & 1u, abort_flag);
-        if (t == 0) mbar_wait_lean(smem_u32(&sh->v_full[vs]), (vit / VST) & 1u, abort_flag);
+        mma_commit_addr(s_full0 + sb * 8u);
+        if ((g & 7) == 7 && *abort_flag) break;
+      }
+    }
+    __syncwarp();
+  } else if (warp == SATC_WARP_PV) {
+    // ------------------------------------------------------------ product issuer (one lane)
+    // O(tile) += P V for the tiles of the codes walk, each as soon as its P tile is complete.
+    if (lane == 0) {
+      constexpr uint32_t IDESC_PV = satc_idesc(Cfg::DP, true);
+      constexpr uint32_t HI = smem_desc_hi(1024, 2);
+      const uint32_t p_lo = smem_desc_lo(smem_u32(sP));
+      const uint32_t v_lo = ((smem_u32(sV) & 0x3FFFFu) >> 4) | ((uint32_t)(SATC_PANEL >> 4) << 16);  // MN-major: block stride
+      const uint32_t p_full0 = smem_u32(&sh->p_full[0]), p_free0 = smem_u32(&sh->p_free[0]);
+      const uint32_t v_full0 = smem_u32(&sh->v_full[0]), v_empty0 = smem_u32(&sh->v_empty[0]);
+      uint32_t pb = 0, p_par = 0, vs = 0, v_par = 0;
+      for (int c = 0; c < per_walk; ++c) {
+        const uint32_t t = NT == 2 ? ((uint32_t)c & 1u) : 0u;
+        mbar_wait_lean(p_full0 + pb * 8u, p_par, abort_flag);
+        if (t == 0) mbar_wait_lean(v_full0 + vs * 8u, v_par, abort_flag);
         tc_fence_after();
+        const uint32_t a_lo = p_lo + pb * (uint32_t)(Cfg::P_TILE >> 4), b_lo = v_lo + vs * (uint32_t)(Cfg::TILE >> 4);
+        const uint32_t d_tmem = tmem_base + SATC_TMEM_O + t * Cfg::DP;
+        const uint32_t acc0 = c >= NT ? 1u : 0u;  // the first key block starts the accumulator
 #pragma unroll
-        for (int kstep = 0; kstep < SATC_BK / 16; ++kstep) {
-          const uint64_t da = smem_desc(p_addr + pb * Cfg::P_TILE + (kstep >> 2) * SATC_PANEL + (kstep & 3) * 32, 1024, 2);
-          const uint64_t db = smem_desc_mn(v_addr + vs * Cfg::TILE + kstep * 2048, SATC_PANEL, 1024);
-          mma_f16(tmem_base + SATC_TMEM_O + t * Cfg::DP, da, db, IDESC_PV, (jj > 0 || kstep > 0) ? 1u : 0u);
-        }
+        for (int kstep = 0; kstep < SATC_BK / 16; ++kstep)
+          mma_f16_lohi(d_tmem, a_lo + (uint32_t)(((kstep >> 2) * SATC_PANEL + (kstep & 3) * 32) >> 4), HI,
+                       b_lo + (uint32_t)((kstep * 2048) >> 4), HI, IDESC_PV, kstep > 0 ? 1u : acc0);
         if (t == NT - 1) {
-          mma_commit(&sh->v_empty[vs]);
-          ++vit;
+          mma_commit_addr(v_empty0 + vs * 8u);
+          if (++vs == (uint32_t)VST) {
+            vs = 0;
+            v_par ^= 1u;
+          }
         }
-        mma_commit(&sh->p_free[pb]);
-      };
-      mbar_wait_lean(smem_u32(&sh->q_full), 0, abort_flag);
-      const int first_code = (N_WALKS - 1) * per_walk;
-      issue_qk(0);
-      for (int g = 0; g < total && !*abort_flag; ++g) {
-        if (g + 1 < total) issue_qk(g + 1);
-        if (g - 1 >= first_code) issue_pv(g - 1 - first_code);
+        mma_commit_addr(p_free0 + pb * 8u);
+        if (++pb == (uint32_t)PST) {
+          pb = 0;
+          p_par ^= 1u;
+        }
+        if ((c & 7) == 7 && *abort_flag) break;
       }
-      if (!*abort_flag) {
-        issue_pv(per_walk - 1);
-        mma_commit(&sh->o_full);
-      }
+      mma_commit_addr(smem_u32(&sh->o_full));
     }
     __syncwarp();
   } else {
