@@ -8,8 +8,8 @@
 // 128 two or three times:
 //   walk "max"   : S = Q K^T into tensor memory, every row keeps its largest logit;
 //   walk "sum"   : (fixed scale only) the row sums of 2^(t - max), which the codes then depend on;
-//   walk "codes" : S again; code = rint(base - t) in the log domain, P = 2^(14 - code) as fp16 into a
-//                  shared-memory operand tile, O += P V on the tensor cores.  With the row maximum as
+//   walk "codes" : S again; code = rint(base - t) in the log domain, P = 2^(14 - code) as fp16 into
+//                  tensor memory, O += P V on the tensor cores with P read from there.  With the row maximum as
 //                  scale the codes do not depend on the row sum, which is then gathered in this walk.
 // Roles: 16 softmax warps (warp w reads tensor-memory lanes 32 (w % 4) .. +31, columns 32 (w / 4) .. +31
 // of every score tile), one TMA producer lane, one lane that issues the score MMAs and one that issues
@@ -45,7 +45,7 @@ constexpr int SATC_THREADS = 19 * 32;
 constexpr int SATC_BQ = 128;            // query rows per tile
 constexpr int SATC_BK = 128;            // keys per block
 constexpr int SATC_PANEL = 128 * 128;   // bytes of one 64-feature (or 64-key) panel of 128 rows
-constexpr int SATC_TMEM_O = 256;        // first column of the output accumulators (score buffers at 0 and 128)
+constexpr int SATC_TMEM_P = 256;        // first column of the P tiles (score buffers at columns 0 and 128)
 
 template <int D>
 struct SaTcCfg {
@@ -53,18 +53,20 @@ struct SaTcCfg {
   static constexpr int NP = (D + 63) / 64;
   static constexpr int NT = NP == 1 ? 2 : 1;   // query tiles per CTA (shared memory and tensor memory budget)
   static constexpr int KSTEPS = DP / 16;
-  static constexpr int KST = NP == 1 ? 3 : (NP == 2 ? 2 : 1);
-  static constexpr int VST = NP == 1 ? 2 : 1;
-  static constexpr int PST = NP <= 2 ? 2 : 1;
+  static constexpr int KST = NP <= 2 ? 3 : 2;
+  static constexpr int VST = NP <= 2 ? 2 : 1;
+  // P = 2^(14 - code) as fp16 lives in tensor memory (64 columns per tile of 128 keys) and is the A
+  // operand of P V from there: two tiles in flight where the accumulators leave room
+  static constexpr int PST = (SATC_TMEM_P + 128 + NT * DP <= 512) ? 2 : 1;
+  static constexpr int TMEM_O = SATC_TMEM_P + PST * 64;
   static constexpr int TILE = NP * SATC_PANEL;
-  static constexpr int P_TILE = 2 * SATC_PANEL;
   static constexpr int OFF_K = NT * TILE;
   static constexpr int OFF_V = OFF_K + KST * TILE;
-  static constexpr int OFF_P = OFF_V + VST * TILE;
-  static constexpr int OFF_SH = OFF_P + PST * P_TILE;
+  static constexpr int OFF_SH = OFF_V + VST * TILE;
   static constexpr int SMEM = 1024 + OFF_SH + 1024 + 2 * 4 * SATC_BQ * 4;
   static_assert(SMEM <= 232448, "shared memory budget");
-  static_assert(SATC_TMEM_O + NT * DP <= 512, "tensor memory budget");
+  static_assert(TMEM_O + NT * DP <= 512, "tensor memory budget");
+  static_assert(NT == 1 || PST == 2, "alternating query tiles need two P tiles");
 };
 
 struct SaTcShared {
@@ -101,6 +103,26 @@ __device__ __forceinline__ void mma_f16_lohi(uint32_t d_tmem, uint32_t a_lo, uin
       ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// A from tensor memory (128 lanes x 8 columns of packed fp16 pairs per K step of 16), B from shared memory.
+__device__ __forceinline__ void mma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi,
+                                           uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// 32 lanes x 16 consecutive 32-bit columns: thread i of the warp writes row (lane base + i).
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 // MN-major operand with 128-byte swizzled rows (one row = 64 contiguous elements of the M/N axis for
 // one k): `lbo` = bytes between 64-element blocks of the M/N axis, `sbo` = bytes between groups of 8 k.
 __device__ __forceinline__ uint64_t smem_desc_mn(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -131,7 +153,6 @@ self_attn_logq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   unsigned char* sQ = smem;
   unsigned char* sK = smem + Cfg::OFF_K;
   unsigned char* sV = smem + Cfg::OFF_V;
-  unsigned char* sP = smem + Cfg::OFF_P;
   SaTcShared* sh = reinterpret_cast<SaTcShared*>(smem + Cfg::OFF_SH);
   float* mpart = reinterpret_cast<float*>(smem + Cfg::OFF_SH + 1024);  // [4][128] partial row maxima
   float* zpart = mpart + 4 * SATC_BQ;                                  // [4][128] partial row sums
@@ -256,7 +277,6 @@ self_attn_logq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     if (lane == 0) {
       constexpr uint32_t IDESC_PV = satc_idesc(Cfg::DP, true);
       constexpr uint32_t HI = smem_desc_hi(1024, 2);
-      const uint32_t p_lo = smem_desc_lo(smem_u32(sP));
       const uint32_t v_lo = ((smem_u32(sV) & 0x3FFFFu) >> 4) | ((uint32_t)(SATC_PANEL >> 4) << 16);  // MN-major: block stride
       const uint32_t p_full0 = smem_u32(&sh->p_full[0]), p_free0 = smem_u32(&sh->p_free[0]);
       const uint32_t v_full0 = smem_u32(&sh->v_full[0]), v_empty0 = smem_u32(&sh->v_empty[0]);
@@ -266,13 +286,13 @@ self_attn_logq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         mbar_wait_lean(p_full0 + pb * 8u, p_par, abort_flag);
         if (t == 0) mbar_wait_lean(v_full0 + vs * 8u, v_par, abort_flag);
         tc_fence_after();
-        const uint32_t a_lo = p_lo + pb * (uint32_t)(Cfg::P_TILE >> 4), b_lo = v_lo + vs * (uint32_t)(Cfg::TILE >> 4);
-        const uint32_t d_tmem = tmem_base + SATC_TMEM_O + t * Cfg::DP;
+        const uint32_t a_tmem = tmem_base + SATC_TMEM_P + pb * 64u, b_lo = v_lo + vs * (uint32_t)(Cfg::TILE >> 4);
+        const uint32_t d_tmem = tmem_base + Cfg::TMEM_O + t * Cfg::DP;
         const uint32_t acc0 = c >= NT ? 1u : 0u;  // the first key block starts the accumulator
 #pragma unroll
         for (int kstep = 0; kstep < SATC_BK / 16; ++kstep)
-          mma_f16_lohi(d_tmem, a_lo + (uint32_t)(((kstep >> 2) * SATC_PANEL + (kstep & 3) * 32) >> 4), HI,
-                       b_lo + (uint32_t)((kstep * 2048) >> 4), HI, IDESC_PV, kstep > 0 ? 1u : acc0);
+          mma_f16_ts(d_tmem, a_tmem + (uint32_t)(kstep * 8), b_lo + (uint32_t)((kstep * 2048) >> 4), HI, IDESC_PV,
+                     kstep > 0 ? 1u : acc0);
         if (t == NT - 1) {
           mma_commit_addr(v_empty0 + vs * 8u);
           if (++vs == (uint32_t)VST) {
@@ -368,14 +388,11 @@ self_attn_logq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             const int64_t code_row =
                 (((int64_t)b * a.H + h) * a.nq + row0 + t * SATC_BQ + row) * a.nk + j * SATC_BK + cp * 32;
             const unsigned long long base2 = pack_f32x2(base[t], base[t]);
-            unsigned char* prow = sP + pb * Cfg::P_TILE + (cp >> 1) * SATC_PANEL + row * 128;
+            uint32_t pk[16];
             unsigned long long zs = zsum2[t];
+            {
 #pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
-              uint32_t pk[4];
-#pragma unroll
-              for (int i2 = 0; i2 < 4; ++i2) {
-                const int i = c4 * 8 + i2 * 2;
+              for (int i = 0; i < 32; i += 2) {
                 // x = base - t * scale >= 0 up to rounding (the row maximum has code 0); -inf logits (keys
                 // beyond nk) give +inf, which the integer minimum below clamps to the last code
                 unsigned long long x2 = fma_f32x2(pack_f32x2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), nscale2, base2);
@@ -399,16 +416,16 @@ self_attn_logq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 const float p0 = __uint_as_float(0x46800000u - (min(b0, p_top) << 23));
                 const float p1 = __uint_as_float(0x46800000u - (min(b1, p_top) << 23));
                 const __half2 ph = __floats2half2_rn(p0, p1);
-                pk[i2] = *reinterpret_cast<const uint32_t*>(&ph);
+                pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&ph);  // key i in the low half
               }
-              if (c4 == 0) {
-                mbar_wait_lean(smem_u32(&sh->p_free[pb]), ((c / PST) & 1u) ^ 1u, abort_flag);
-                __syncwarp();
-              }
-              *reinterpret_cast<uint4*>(prow + ((((cp & 1) * 4 + c4) ^ (row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
             }
             zsum2[t] = zs;
-            fence_proxy_async_smem();
+            // the P tile's previous product must have read it
+            mbar_wait_lean(smem_u32(&sh->p_free[pb]), ((c / PST) & 1u) ^ 1u, abort_flag);
+            __syncwarp();
+            tmem_st16(t_lane + SATC_TMEM_P + pb * 64u + cp * 16u, pk);
+            tmem_st_wait();
+            tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh->p_full[pb]);
             ++c;
@@ -464,7 +481,7 @@ self_attn_logq_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       __half* o_row = a.O + (((int64_t)b * a.nq + orow) * a.H + h) * D;
       for (int ch = cp; ch < D / 8; ch += 4) {
         uint32_t o[8];
-        tmem_ld8(t_lane + SATC_TMEM_O + t * Cfg::DP + ch * 8, o);
+        tmem_ld8(t_lane + Cfg::TMEM_O + t * Cfg::DP + ch * 8, o);
         tmem_ld_wait();
         __half2 oh[4];
 #pragma unroll
