@@ -27,6 +27,13 @@ def _sample_rows(M, seed):
     (4096, 2, 1280, 320, 8),     # FF2: long K, two column blocks
     (4096, 2, 320, 960, 8),      # stacked q/k/v projection
     (1024, 8, 640, 640, 4),      # 32 x 32 level, 4-bit weights
+    # 4-bit weights over every transformer linear of the four UNet levels at batch 8: q/k/v/out (ch -> ch),
+    # the gated feed-forward (ch -> 8 ch, 4 ch -> ch) and the cross-attention k/v projections of the 77
+    # context tokens (768 -> ch)
+    (4096, 8, 320, 320, 4), (4096, 8, 320, 2560, 4), (4096, 8, 1280, 320, 4), (77, 8, 768, 320, 4),
+    (1024, 8, 640, 5120, 4), (1024, 8, 2560, 640, 4), (77, 8, 768, 640, 4),
+    (256, 8, 1280, 1280, 4), (256, 8, 1280, 10240, 4), (256, 8, 5120, 1280, 4), (77, 8, 768, 1280, 4),
+    (64, 8, 1280, 1280, 4), (64, 8, 1280, 10240, 4), (64, 8, 5120, 1280, 4),
 ])
 def test_linear_full_size_sampled_rows(P, batch, C, N, w_bits):
     torch, b = gpu()
@@ -54,10 +61,15 @@ def test_linear_full_size_sampled_rows(P, batch, C, N, w_bits):
     assert np.isfinite(Y.float().cpu().numpy()).all()            # every tile was written
 
 
-def test_conv_full_size_sampled_bands():
-    """2 x 64 x 64 x 320 -> 320, W4A6, 16 groups: image-border and interior bands of output rows."""
+@pytest.mark.parametrize("n,H,Wd,C", [
+    (2, 64, 64, 320),            # the benchmark's launch
+    (8, 64, 64, 320), (8, 32, 32, 640), (8, 16, 16, 1280), (8, 8, 8, 1280),   # the four levels at batch 8
+])
+def test_conv_full_size_sampled_bands(n, H, Wd, C):
+    """3 x 3 conv C -> C, W4A6, 16 groups: image-border and interior bands of output rows of the first, second
+    and last image."""
     torch, b = gpu()
-    n, H, Wd, C, N, K = 2, 64, 64, 320, 320, 16
+    N, K = C, 16
     P = H * Wd
     Xcal = synth.activations(22, 100, 4, P, C, None, None, token_outliers=False)
     X = synth.activations(22, 1, n, P, C, None, None, token_outliers=False)
@@ -76,7 +88,9 @@ def test_conv_full_size_sampled_bands():
     codes, _, _ = ol.quantize_static(X, gr, 0)
     codes = codes.reshape(n, H, Wd, C)
     worst, ref_max = 0.0, 0.0
-    for img, h0, h1 in [(0, 0, 2), (0, 31, 33), (0, 62, 64), (1, 0, 1), (1, 1, 3), (1, 63, 64)]:
+    mid = H // 2
+    for img, h0, h1 in [(0, 0, 2), (0, mid - 1, mid + 1), (0, H - 2, H), (1, 0, 1), (1, 1, 3), (1, H - 1, H),
+                        (n - 1, 0, 1), (n - 1, mid, mid + 1), (n - 1, H - 1, H)]:
         lo, hi = max(h0 - 1, 0), min(h1 + 1, H)                  # the band with the rows it reads
         sub = ol.group_conv3x3(codes[img:img + 1, lo:hi], gr.scale[0][0], gr.zp[0][0], gr.col_group, wq, sw, bias)
         ref = sub[0, h0 - lo:h0 - lo + (h1 - h0)]                # rows whose neighbours are real rows or the border
@@ -86,11 +100,14 @@ def test_conv_full_size_sampled_bands():
     assert np.isfinite(Yg).all()
 
 
-def test_attention_full_size():
-    """B 2, H 8, nq 4096, nk 77, d 40, 8-bit codes: the whole output against the oracle."""
+@pytest.mark.parametrize("nq,d,bits", [(4096, 40, 8), (4096, 40, 4), (1024, 80, 8), (256, 160, 8), (64, 160, 8),
+                                       (64, 160, 4)])
+def test_attention_full_size(nq, d, bits):
+    """B 2, H 8, nk 77 at the four UNet levels (nq x d = 4096 x 40 ... 64 x 160): the whole output against
+    the oracle."""
     torch, b = gpu()
-    Q, K, V = synth.attention_inputs(23, 2, 8, 4096, 77, 40)
-    _compare(torch, b, Q, K, V, 8)
+    Q, K, V = synth.attention_inputs(23, 2, 8, nq, 77, d)
+    _compare(torch, b, Q, K, V, bits)
 
 
 def test_self_attention_full_size_sampled_rows():
