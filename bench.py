@@ -543,6 +543,8 @@ MICRO_CASES = {
     "attn_qv_2x4096x40": ("attn", dict(B=2, H=8, nq=4096, nk=77, d=40, v_bits=8)),
     "attn_8x1024x80": ("attn", dict(B=8, H=8, nq=1024, nk=77, d=80)),
     "attn_8x256x160": ("attn", dict(B=8, H=8, nq=256, nk=77, d=160)),
+    "attn_sdxl_1x10x1024x64": ("attn", dict(B=1, H=10, nq=1024, nk=77, d=64)),
+    "gemm_sdxl_1024x5120x640_w8": ("gemm", dict(M=1024, P=1024, N=5120, C=640, G=8, wbits=8)),
     "selfattn_2x4096x40": ("selfattn", dict(B=2, H=8, n=4096, d=40)),
     "selfattn_8x1024x80": ("selfattn", dict(B=8, H=8, n=1024, d=80)),
     "selfattn_8x256x160": ("selfattn", dict(B=8, H=8, n=256, d=160)),

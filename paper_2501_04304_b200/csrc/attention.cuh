@@ -269,15 +269,19 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_phase2_kernel(const AttnAr
   uint4 xk[KStage<D, NKP>::N];
   load_k<D, NKP>(a, b, h, xk);
   // V^T: 128-bit loads of 8 features of one key, written transposed; keys >= nk and key 0 are zero.
-  // K, V and Q are all requested before anything is written, so their latencies overlap.
+  // Consecutive lanes take consecutive keys of the same 8 features, so that the transposed 2-byte stores
+  // of a warp fall into consecutive words of one V^T row (the head's V slab is a few KB and sits in L2,
+  // so the strided reads cost little).  K, V and Q are all requested before anything is written, so
+  // their latencies overlap.
   constexpr int NV = (NKP * 16 * (D / 8) + AT_THREADS - 1) / AT_THREADS;
   uint4 xv[NV];
 #pragma unroll
   for (int e = 0; e < NV; ++e) {
     const int i = threadIdx.x + e * AT_THREADS;
-    const int j = i / (D / 8), v = i - j * (D / 8);
+    const int v = i / (NKP * 16), j = i - v * (NKP * 16);
     xv[e] = make_uint4(0, 0, 0, 0);
-    if (j < a.nk) xv[e] = __ldg(reinterpret_cast<const uint4*>(a.V + (((int64_t)b * a.nk + j) * a.H + h) * D) + v);
+    if (j < a.nk && v < D / 8)
+      xv[e] = __ldg(reinterpret_cast<const uint4*>(a.V + (((int64_t)b * a.nk + j) * a.H + h) * D) + v);
   }
   if (rows_valid > 0) stage_q<D, NKP>(a.Q + (((int64_t)b * a.nq + row0) * a.H + h) * D, q_stride, rows_valid, slab);
   store_k<D, NKP>(xk, sK);
@@ -291,7 +295,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_phase2_kernel(const AttnAr
 #pragma unroll
     for (int ev = 0; ev < NV; ++ev) {
       const int i = threadIdx.x + ev * AT_THREADS;
-      if (i / (D / 8) < a.nk) {
+      if (i % (NKP * 16) < a.nk && i < NKP * 16 * (D / 8)) {
         const __half* xh = reinterpret_cast<const __half*>(&xv[ev]);
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
@@ -325,7 +329,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_phase2_kernel(const AttnAr
   for (int ev = 0; ev < NV; ++ev) {
     const int i = threadIdx.x + ev * AT_THREADS;
     if (i >= NKP * 16 * (D / 8)) continue;
-    const int j = i / (D / 8), v = i - j * (D / 8);
+    const int v = i / (NKP * 16), j = i - v * (NKP * 16);
     const __half* xh = reinterpret_cast<const __half*>(&xv[ev]);
     float f[8];
 #pragma unroll

@@ -34,6 +34,10 @@ def _sample_rows(M, seed):
     (1024, 8, 640, 5120, 4), (1024, 8, 2560, 640, 4), (77, 8, 768, 640, 4),
     (256, 8, 1280, 1280, 4), (256, 8, 1280, 10240, 4), (256, 8, 5120, 1280, 4), (77, 8, 768, 1280, 4),
     (64, 8, 1280, 1280, 4), (64, 8, 1280, 10240, 4), (64, 8, 5120, 1280, 4),
+    # the second model of Table 2 (SDXL-Turbo at 512 x 512, one image): transformer levels of 1024 tokens x
+    # 640 channels and 256 tokens x 1280 channels, context of 77 tokens x 2048
+    (1024, 1, 640, 640, 8), (1024, 1, 640, 5120, 8), (1024, 1, 2560, 640, 8), (77, 1, 2048, 640, 8),
+    (256, 1, 1280, 1280, 8), (256, 1, 1280, 10240, 4), (256, 1, 5120, 1280, 4), (77, 1, 2048, 1280, 4),
 ])
 def test_linear_full_size_sampled_rows(P, batch, C, N, w_bits):
     torch, b = gpu()
@@ -108,6 +112,14 @@ def test_attention_full_size(nq, d, bits):
     torch, b = gpu()
     Q, K, V = synth.attention_inputs(23, 2, 8, nq, 77, d)
     _compare(torch, b, Q, K, V, bits)
+
+
+@pytest.mark.parametrize("H,nq", [(10, 1024), (20, 256)])
+def test_attention_sdxl_turbo_levels(H, nq):
+    """Heads of 64 features (640 / 10 and 1280 / 20 channels), context projected from 2048 features."""
+    torch, b = gpu()
+    Q, K, V = synth.attention_inputs(24, 1, H, nq, 77, 64, ctx_dim=2048)
+    _compare(torch, b, Q, K, V, 8)
 
 
 def test_self_attention_full_size_sampled_rows():
