@@ -220,14 +220,15 @@ dgq_status dgq_cross_attn_workspace_bytes(int B, int H, int nq, int nk, int d, s
  *     starting any stream capture.  Later calls only enqueue work on `stream`;
  *   - the call itself performs no allocation and frees nothing;
  *   - all calls on a device share the one array.  It still holds the previous
- *     call's statistics on entry; the part that must start clean is reset on
- *     `stream` before the kernels run.  Two calls whose kernels can overlap on the
- *     GPU (different streams without an ordering between them) race on it:
+ *     call's statistics on entry; nothing in it has to start clean, because the
+ *     first kernel writes every entry that the second one reads.  Two calls whose
+ *     kernels can overlap on the GPU (different streams without an ordering
+ *     between them) race on it:
  *     serialise them, or use dgq_cross_attn_logq with separate workspaces.
  * Errors: those of dgq_cross_attn_logq. */
 #define DGQ_NOALLOC_MAX_ROWS (1 << 18)
 #define DGQ_NOALLOC_MAX_HEADS 256
-#define DGQ_NOALLOC_SCRATCH_BYTES (1024 + 8 * DGQ_NOALLOC_MAX_ROWS)
+#define DGQ_NOALLOC_SCRATCH_BYTES (4 * (DGQ_NOALLOC_MAX_ROWS / 128 + DGQ_NOALLOC_MAX_HEADS) + 8 * DGQ_NOALLOC_MAX_ROWS)
 dgq_status dgq_cross_attn_logq_noalloc(const void* Q, const void* K, const void* V, int B, int H, int nq, int nk,
                                        int d, int score_bits, int scale_gran, const float* fixed_scale, void* O,
                                        float* scale_out, uint8_t* codes_out, void* stream);

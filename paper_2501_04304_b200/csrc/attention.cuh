@@ -4,8 +4,11 @@
 // is two kernels on one stream:
 //   phase 1  logits Q K^T (tensor cores, fp32 accumulate), per-row softmax statistics
 //            (row maximum and log2 of the row sum, in base-2 logits) and the largest
-//            off-<start> log2-score of the scope, reduced with an ordered-integer atomicMax;
-//   phase 2  the same logits again (bit-identical), codes in the log domain
+//            off-<start> log2-score of the CTA's rows, one partial maximum per CTA (no atomics,
+//            nothing to initialise: every partial is written before the next kernel reads it);
+//   phase 2  the scale of the scope = the largest of its CTAs' partial maxima (a contiguous run
+//            of at most B H ceil(nq / rows per CTA) floats, read once per CTA from L2);
+//            the same logits again (bit-identical), codes in the log domain
 //            code = clamp(rint(log2 s - log2 A_ij), 0, 2^b - 1) with no transcendental per score,
 //            2^-code built by writing the exponent field, A_hat V on tensor cores, and the
 //            <start> column added as a separate fp32 rank-1 term A_i0 V_0.
@@ -50,7 +53,7 @@ struct AttnArgs {
   int B, H, nq, nk, d, bits, gran;
   int v_bits;              // 0: V as given; else V_hat = linear quantizer (Eq. 1, Eq. 6) over the head's [nk, d] slab
   float qk_scale_log2;     // log2(e) / sqrt(d)
-  int* smax;               // workspace: ordered-int log2 of the scale per scope
+  float* part;             // workspace: log2 of the largest off-<start> score of every phase-1 CTA [B][H][row blocks]
   float2* stats;           // workspace: (row max, log2 row sum) [B][H][nq]
   const float* fixed_scale;
   float* scale_out;
@@ -241,8 +244,14 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_phase1_kernel(const AttnAr
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, o));
-  if (lane == 0 && best > -INFINITY && a.fixed_scale == nullptr)
-    atomicMax(&a.smax[scope_index(a, b, h)], float_to_ordered(best));
+  __shared__ float best_w[AT_WARPS];
+  if (lane == 0) best_w[warp] = best;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+#pragma unroll
+    for (int w = 1; w < AT_WARPS; ++w) best = fmaxf(best, best_w[w]);
+    a.part[((int64_t)b * a.H + h) * a.n_row_blocks + rb] = best;
+  }
 }
 
 template <int D, int NKP, bool CODES>
@@ -282,6 +291,21 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_phase2_kernel(const AttnAr
     xv[e] = make_uint4(0, 0, 0, 0);
     if (j < a.nk && v < D / 8)
       xv[e] = __ldg(reinterpret_cast<const uint4*>(a.V + (((int64_t)b * a.nk + j) * a.H + h) * D) + v);
+  }
+  // The scope's scale: its CTAs' partial maxima lie next to each other (row blocks of a head, heads of a
+  // prompt, prompts of the call); each thread takes a strided share, the warps meet after the barrier below.
+  __shared__ float part_w[AT_WARPS];
+  if (!a.fixed_scale) {
+    const int per_head = a.n_row_blocks;
+    const int64_t first = a.gran == DGQ_SCALE_PER_PROMPT ? (int64_t)b * a.H * per_head
+                          : (a.gran == DGQ_SCALE_PER_PROMPT_HEAD ? ((int64_t)b * a.H + h) * per_head : 0);
+    const int count = a.gran == DGQ_SCALE_PER_PROMPT ? a.H * per_head
+                      : (a.gran == DGQ_SCALE_PER_PROMPT_HEAD ? per_head : a.B * a.H * per_head);
+    float m = -INFINITY;
+    for (int i = threadIdx.x; i < count; i += AT_THREADS) m = fmaxf(m, __ldg(a.part + first + i));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0) part_w[warp] = m;
   }
   if (rows_valid > 0) stage_q<D, NKP>(a.Q + (((int64_t)b * a.nq + row0) * a.H + h) * D, q_stride, rows_valid, slab);
   store_k<D, NKP>(xk, sK);
@@ -352,10 +376,13 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_phase2_kernel(const AttnAr
   __syncthreads();
   const int scope = scope_index(a, b, h);
   float log2s;
-  if (a.fixed_scale)
+  if (a.fixed_scale) {
     log2s = log2f(fmaxf(__ldg(a.fixed_scale + scope), 1.17549435e-38f));
-  else
-    log2s = ordered_to_float(a.smax[scope]);
+  } else {
+    log2s = part_w[0];
+#pragma unroll
+    for (int w = 1; w < AT_WARPS; ++w) log2s = fmaxf(log2s, part_w[w]);
+  }
   if (a.scale_out && threadIdx.x == 0 && rb == 0 &&
       (a.gran == DGQ_SCALE_PER_PROMPT_HEAD || (a.gran == DGQ_SCALE_PER_PROMPT && h == 0) || (b == 0 && h == 0)))
     a.scale_out[scope] = exp2f(log2s);
@@ -475,13 +502,16 @@ static dgq_status launch_attn_d(const AttnArgs& a, cudaStream_t stream) {
   return launch_attn<D, 8>(a, stream);
 }
 
-static size_t attn_smax_bytes(int B, int H) { return ((size_t)B * H * sizeof(int) + 255) / 256 * 256; }
+// One partial maximum per phase-1 CTA; the bound holds for every kernel configuration (128 or 256 rows per CTA).
+static size_t attn_part_bytes(int B, int H, int nq) {
+  return ((size_t)B * H * ((nq + 127) / 128) * sizeof(float) + 255) / 256 * 256;
+}
 
 }  // namespace dgq
 
 extern "C" dgq_status dgq_cross_attn_workspace_bytes(int B, int H, int nq, int nk, int d, size_t* bytes) {
   if (!bytes || B <= 0 || H <= 0 || nq <= 0 || nk < 2 || d <= 0) return DGQ_ERR_INVALID_ARG;
-  *bytes = dgq::attn_smax_bytes(B, H) + (size_t)B * H * nq * sizeof(float2);
+  *bytes = dgq::attn_part_bytes(B, H, nq) + (size_t)B * H * nq * sizeof(float2);
   return DGQ_OK;
 }
 
@@ -515,15 +545,13 @@ static dgq_status attn_run(const void* Q, const void* K, const void* V, int B, i
   a.gran = scale_gran;
   a.v_bits = v_bits;
   a.qk_scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)d));
-  a.smax = (int*)workspace;
-  a.stats = (float2*)((char*)workspace + attn_smax_bytes(B, H));
+  a.part = (float*)workspace;
+  a.stats = (float2*)((char*)workspace + attn_part_bytes(B, H, nq));
   a.fixed_scale = fixed_scale;
   a.scale_out = scale_out;
   a.codes_out = codes_out;
   a.n_row_blocks = 0;  // set per kernel configuration at launch
   cudaStream_t st = (cudaStream_t)stream;
-  // 0x80 bytes decode to about -3.4e38 in the ordered-integer encoding: "no score seen yet"
-  DGQ_CUDA_OK(cudaMemsetAsync(a.smax, 0x80, attn_smax_bytes(B, H), st));
   switch (d) {
     case 40: return launch_attn_d<40>(a, st);
     case 64: return launch_attn_d<64>(a, st);

@@ -43,8 +43,8 @@ extern "C" dgq_status dgq_cross_attn_logq_noalloc(const void* Q, const void* K, 
     }
     scratch = g_noalloc_ptr[dev];
   }
-  // The workspace path resets the per-scope maxima on `stream` itself and overwrites every row
-  // statistic it later reads, so stale contents from an earlier call are harmless.
+  // The first kernel of the workspace path writes every partial maximum and every row statistic
+  // that the second one reads, so stale contents from an earlier call are harmless.
   return dgq_cross_attn_logq(Q, K, V, B, H, nq, nk, d, score_bits, scale_gran, fixed_scale, O, scale_out,
                              codes_out, scratch, (size_t)DGQ_NOALLOC_SCRATCH_BYTES, stream);
 }
