@@ -59,17 +59,25 @@ constexpr int GEMM_MAX_ATOMS = 1024;           // 32768 reduction positions
 constexpr int GEMM_A_STAGE = GEMM_BM * 128;  // bytes
 constexpr int GEMM_SMEM_LIMIT = 227 * 1024;
 
-template <int BN>
+template <int BN, bool W4>
 struct GemmCfg {
+  // 4-bit weights: ring of packed B stages (BN rows x 64 bytes each) that the unpack warps fill with
+  // asynchronous copies PK_AHEAD stages ahead of the stage they expand
+  static constexpr int PK_STAGES = W4 ? 4 : 0;
+  static constexpr int PK_AHEAD = PK_STAGES - 1;
+  static constexpr int PK_STAGE = BN * 64;
+  static constexpr int PK_BYTES = PK_STAGES * PK_STAGE;
   static constexpr int B_STAGE = BN * 128;
   static constexpr int STAGE = GEMM_A_STAGE + B_STAGE;
   static constexpr int OUT_BYTES = GEMM_BM * BN * 2;  // fp16 staging of one output tile
   static constexpr int MISC_BYTES = 2048 + (2 + DGQ_MAX_GROUPS) * BN * 4 + GEMM_MAX_ATOMS * 4;  // barriers + sw, bias, wsum of the CTA's columns + conv atom table
-  static constexpr int STAGES_RAW = (GEMM_SMEM_LIMIT - 1024 - OUT_BYTES - MISC_BYTES) / STAGE;
+  static constexpr int STAGES_RAW = (GEMM_SMEM_LIMIT - 1024 - OUT_BYTES - MISC_BYTES - PK_BYTES) / STAGE;
   static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
   static constexpr int NACC_RAW = 512 / BN;
   static constexpr int NACC = NACC_RAW > 4 ? 4 : NACC_RAW;
-  static constexpr int SMEM = STAGES * STAGE + OUT_BYTES + MISC_BYTES + 1024;
+  static constexpr int OFF_PK = STAGES * STAGE + OUT_BYTES + MISC_BYTES;
+  static constexpr int SMEM = OFF_PK + PK_BYTES + 1024;
+  static_assert(MISC_BYTES % 16 == 0, "the packed ring is 16-byte aligned");
   static_assert(BN % 32 == 0 && BN <= 256, "BN must be a multiple of 32 up to 256");
   static_assert(NACC >= 2, "need two accumulators to overlap the epilogue");
   static_assert(NACC * BN <= 512, "tensor memory has 512 columns");
@@ -116,7 +124,7 @@ template <int BN, bool W4, bool CONV>
 __global__ void __maxnreg__(gemm_regs_launch(W4))
 gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmY, const __grid_constant__ GemmArgs a) {
-  using Cfg = GemmCfg<BN>;
+  using Cfg = GemmCfg<BN, W4>;
   constexpr int STAGES = Cfg::STAGES;
   constexpr int NACC = Cfg::NACC;
   extern __shared__ unsigned char smem_dyn[];
@@ -324,27 +332,45 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncwarp();
   } else if (W4 && warp >= GEMM_WARP_STORE + 1) {
     // ------------------------------------------------------------ 4-bit weight unpack into the B stage
+    // Every thread owns the same 16-byte pieces of every stage.  It copies them asynchronously from global
+    // memory into its slots of the packed ring PK_AHEAD stages before it expands them, one copy group per
+    // stage, and reads back only what it copied itself, so the ring needs no barrier: waiting for its own
+    // copy groups is enough.  The load latency (L2 or DRAM) is thus spread over PK_AHEAD stages.
     constexpr int ITEMS = (BN * 4 + GEMM_UNPACK_THREADS - 1) / GEMM_UNPACK_THREADS;  // 16-byte pieces per thread
+    constexpr int AHEAD = Cfg::PK_AHEAD;
     const int ut = threadIdx.x - GEMM_THREADS_W8;  // 0..GEMM_UNPACK_THREADS-1
+    unsigned char* pk_ring = smem + Cfg::OFF_PK;
     uint32_t it = 0;
     bool ok = true;
     const int row_bytes = a.Kt >> 1;
-    uint4 pk[ITEMS];
-    auto fetch = [&](int tile, int ks) {
-      const int n0 = (tile % a.n_tiles_n) * BN;
+    int f_tile = blockIdx.x, f_ks = 0;  // next stage to request
+    uint32_t f_it = 0;
+    auto request_next = [&]() {
+      if (f_tile < n_tiles) {
+        const int n0 = (f_tile % a.n_tiles_n) * BN;
+        const uint32_t slot = smem_u32(pk_ring + (f_it % Cfg::PK_STAGES) * Cfg::PK_STAGE);
 #pragma unroll
-      for (int e = 0; e < ITEMS; ++e) {
-        const int item = ut + e * GEMM_UNPACK_THREADS;
-        const int r = item >> 2, qd = item & 3;  // B row, 16-byte packed quarter of the 64-byte row slice
-        const int kb = ks * 64 + qd * 16;
-        pk[e] = make_uint4(0u, 0u, 0u, 0u);
-        if (item < BN * 4 && kb < row_bytes)
-          pk[e] = __ldg(reinterpret_cast<const uint4*>(a.w_packed + (size_t)(n0 + r) * row_bytes + kb));
+        for (int e = 0; e < ITEMS; ++e) {
+          const int item = ut + e * GEMM_UNPACK_THREADS;
+          if (item >= BN * 4) continue;
+          const int r = item >> 2, qd = item & 3;  // B row, 16-byte packed quarter of the 64-byte row slice
+          const int kb = f_ks * 64 + qd * 16;
+          const bool in = kb < row_bytes;          // beyond the row: the slot is filled with zeros
+          const uint8_t* src = a.w_packed + (size_t)(n0 + r) * row_bytes + (in ? kb : 0);
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(slot + (uint32_t)item * 16u), "l"(src),
+                       "r"(in ? 16 : 0)
+                       : "memory");
+        }
+        ++f_it;
+        if (++f_ks == n_kstages) {
+          f_ks = 0;
+          f_tile += gridDim.x;
+        }
       }
+      asm volatile("cp.async.commit_group;" ::: "memory");  // one group per call, empty at the end
     };
     // The CTA's whole column block of packed weights (BN rows of Kt / 2 bytes) is asked into L2 up
-    // front: the register look-ahead below is one stage deep, which covers an L2 hit but not a
-    // trip to DRAM.
+    // front, so that the copies below find it there.
     if ((int)blockIdx.x < n_tiles) {
       const int n0 = ((int)blockIdx.x % a.n_tiles_n) * BN;
       const int lines_per_row = (row_bytes + 127) >> 7;
@@ -353,20 +379,25 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const uint8_t* ptr = a.w_packed + (size_t)(n0 + r) * row_bytes + (size_t)l * 128;
         asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
       }
-      fetch(blockIdx.x, 0);
     }
+#pragma unroll
+    for (int i = 0; i < AHEAD; ++i) request_next();
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
       for (int ks = 0; ks < n_kstages && ok; ++ks, ++it) {
+        // the slot of stage it + AHEAD is the one this thread read in the previous iteration
+        request_next();
+        asm volatile("cp.async.wait_group %0;" ::"n"(AHEAD) : "memory");  // this thread's pieces of stage `it` have landed
         const int s = it % STAGES;
         ok = __all_sync(0xffffffffu, mbar_wait(&sh->empty[s], ((it / STAGES) & 1) ^ 1, abort_flag));
         if (!ok) break;
         unsigned char* bst = smB + s * Cfg::B_STAGE;
+        const unsigned char* pst = pk_ring + (it % Cfg::PK_STAGES) * Cfg::PK_STAGE;
 #pragma unroll
         for (int e = 0; e < ITEMS; ++e) {
           const int item = ut + e * GEMM_UNPACK_THREADS;
           if (item >= BN * 4) continue;
           const int r = item >> 2, qd = item & 3;
-          const uint4 p4 = pk[e];
+          const uint4 p4 = *reinterpret_cast<const uint4*>(pst + item * 16);
           const uint4 c0 = make_uint4((p4.x << 4) & 0xF0F0F0F0u, p4.x & 0xF0F0F0F0u, (p4.y << 4) & 0xF0F0F0F0u,
                                       p4.y & 0xF0F0F0F0u);
           const uint4 c1 = make_uint4((p4.z << 4) & 0xF0F0F0F0u, p4.z & 0xF0F0F0F0u, (p4.w << 4) & 0xF0F0F0F0u,
@@ -379,11 +410,9 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh->full[s]);
-        // the next stage's nibbles travel while the tensor core works on this one
-        if (ks + 1 < n_kstages) fetch(tile, ks + 1);
-        else if (tile + (int)gridDim.x < n_tiles) fetch(tile + gridDim.x, 0);
       }
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");  // nothing of this thread's is in flight when the CTA ends
   }
   } else {
     reg_alloc<gemm_regs_epi(W4)>();
@@ -595,7 +624,7 @@ static bool encode_map(CUtensorMap* m, const void* base, int rank, const uint64_
 template <int BN, bool W4, bool CONV>
 static dgq_status launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
                               const GemmArgs& a, int grid, cudaStream_t stream) {
-  using Cfg = GemmCfg<BN>;
+  using Cfg = GemmCfg<BN, W4>;
   static bool attr_set[64] = {false};
   int dev = 0;
   DGQ_CUDA_OK(cudaGetDevice(&dev));
