@@ -108,3 +108,42 @@ def test_centred_layout_and_errors():
     with pytest.raises(b.DgqError) as e:       # misaligned base pointer
         b.quantize_act(g, Xd.view(-1)[4:4 + 64 * 4].view(4, 64))
     assert e.value.status == 2
+
+
+def test_dynamic_token_degenerate_rows():
+    """Rows whose groups are degenerate: all zeros, one constant (near and far from zero), the largest fp16
+    magnitudes, a single spike.  A constant group takes the floor scale, so its zero-point leaves the code
+    range (and, far from zero, the range where the kernel's conversion-free code path applies); codes, scales
+    and zero-points must still match bit for bit, and the layer output must stay within tolerance through the
+    epilogue's zero-point correction."""
+    torch, b = gpu()
+    M, C, N, K = 64, 320, 160, 4
+    Xcal, X, W, bias, gr = layer_case(7, 1, M, C, N, K, 8, oc.DIM_CHANNEL)
+    X = X.copy()
+    X[0] = 0.0
+    X[1] = 3.0
+    X[2] = -5.0
+    X[3] = 65504.0
+    X[4] = -65504.0
+    X[5] = 0.0
+    X[5, 17] = 1000.0
+    X[6, gr.col_group == 0] = 0.25                  # one constant group in an otherwise ordinary row
+    X[7] = 6.1e-5                                   # the smallest normal fp16
+    g = b.calibrate_groups(to_dev(torch, Xcal), M, 8, K, b.DIM_CHANNEL)
+    ref, s_ref, z_ref = ol.quantize_dynamic_token(X, gr.col_group, gr.G, 8)
+    Xq, ds, dz = b.quantize_act(g, to_dev(torch, X), mode=b.MODE_DYNAMIC_TOKEN)
+    assert np.array_equal(ds.cpu().numpy(), s_ref)
+    assert np.array_equal(dz.cpu().numpy(), z_ref)
+    assert np.array_equal(unpermute_codes(Xq, g.export()["perm"], C), ref)
+    wq, sw = ol.weight_rtn(W, 8)
+    w = b.weight_prepare(g, to_dev(torch, W), 8)
+    Y = b.linear(g, w, Xq, mode=b.MODE_DYNAMIC_TOKEN, dyn_scale=ds, dyn_zp=dz, bias=to_dev(torch, bias))
+    assert b.device_status() == 0
+    Yref = ol.group_linear(ref, s_ref, z_ref, gr.col_group, wq, sw, bias)
+    Yg = Y.float().cpu().numpy().astype(np.float64)
+    ordinary = np.ones(M, bool)
+    ordinary[[3, 4]] = False                        # outputs beyond the fp16 range are compared apart
+    assert np.max(np.abs(Yg[ordinary] - Yref[ordinary])) <= 1e-3 * np.max(np.abs(Yref[ordinary]))
+    big = np.clip(Yref[~ordinary], -65504.0, 65504.0)
+    got = np.nan_to_num(Yg[~ordinary], posinf=65504.0, neginf=-65504.0)
+    assert np.max(np.abs(got - big)) <= 1e-3 * np.max(np.abs(big))
