@@ -80,6 +80,26 @@ def test_wide_logits_saturate_four_bits():
         _compare(torch, b, Q, K, V, bits, code_frac=1e-3)
 
 
+def test_uniform_and_one_hot_scores():
+    """Degenerate softmax rows.  Q = 0 gives every key the score 1 / nk: the scale is 1 / nk, every code is 0
+    and the output is the mean of V.  A <start> logit far above the rest leaves the other columns a total
+    weight of about e^-60: the scale follows them down to about 2.5e-26, the codes stay small relative to it
+    and the output is V[0]."""
+    torch, b = gpu()
+    Q, K, V = synth.attention_inputs(12, 2, 2, 200, 77, 40, ctx_dim=64)
+    Q0 = np.zeros_like(Q)
+    O_ref, codes_ref, s_ref, _ = oa.cross_attn_logq(Q0, K, V, 8)
+    assert codes_ref.max() == 0 and np.allclose(s_ref, 1.0 / 77)
+    assert np.allclose(O_ref, V.astype(np.float64).mean(axis=1)[:, None], rtol=0, atol=1e-12)
+    _compare(torch, b, Q0, K, V, 8)
+    K1 = K.copy()
+    K1[:, 0, :, -1] = np.float16(60.0 * np.sqrt(40))      # the <start> column gets e^60 times the others' weight
+    O_ref, codes_ref, _, _ = oa.cross_attn_logq(Q, K1, V, 4)
+    assert np.allclose(O_ref, V[:, :1].astype(np.float64), rtol=0, atol=1e-6)
+    _compare(torch, b, Q, K1, V, 4, code_frac=1e-3)
+    _compare(torch, b, Q, K1, V, 8, code_frac=1e-3)
+
+
 def test_argument_errors():
     torch, b = gpu()
     Q, K, V = synth.attention_inputs(8, 1, 1, 16, 4, 40, ctx_dim=16)
