@@ -168,14 +168,22 @@ __device__ __forceinline__ void logits_warp(const AttnArgs& a, const __half* sla
     }
   }
 #pragma unroll
-  for (int mt = 0; mt < Cfg::MT; ++mt)
+  for (int nt = 0; nt < Cfg::NT; ++nt) {
+    if (nt * 8 + 8 <= a.nk) {  // the whole 8-key tile is real (the same answer in every lane)
 #pragma unroll
-    for (int nt = 0; nt < Cfg::NT; ++nt)
+      for (int mt = 0; mt < Cfg::MT; ++mt)
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int key = nt * 8 + 2 * c + (i & 1);
-        S[mt][nt][i] = key < a.nk ? S[mt][nt][i] * a.qk_scale_log2 : -INFINITY;
-      }
+        for (int i = 0; i < 4; ++i) S[mt][nt][i] *= a.qk_scale_log2;
+    } else {
+#pragma unroll
+      for (int mt = 0; mt < Cfg::MT; ++mt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int key = nt * 8 + 2 * c + (i & 1);
+          S[mt][nt][i] = key < a.nk ? S[mt][nt][i] * a.qk_scale_log2 : -INFINITY;
+        }
+    }
+  }
 }
 
 template <int D, int NKP>
@@ -413,15 +421,18 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_phase2_kernel(const AttnAr
           // rint by adding 1.5 * 2^23: the low bits of the sum are the integer.  -inf logits (padding
           // keys) clamp to the cap; their V^T columns are zero, as is the <start> column.
           const float x = fminf(fmaxf(base - t, 0.f), CODES ? Lf : Lcap);
-          const int code = __float_as_int(x + 12582912.0f) - 0x4B400000;
+          const uint32_t bits = __float_as_uint(x + 12582912.0f);  // 0x4B400000 + code
           if (CODES) {
             const int key = nt * 8 + 2 * c + i;
             const int orow = mt * 16 + r + hi * 8;
             if (key >= 1 && key < a.nk && orow < rows_valid)
-              a.codes_out[(((int64_t)b * a.H + h) * a.nq + row0 + orow) * (a.nk - 1) + key - 1] = (uint8_t)code;
+              a.codes_out[(((int64_t)b * a.H + h) * a.nq + row0 + orow) * (a.nk - 1) + key - 1] = (uint8_t)(bits & 0xFFu);
           }
-          // 2^(14 - code) as an fp32 exponent field; beyond the cap it converts to an fp16 zero
-          p[i] = __int_as_float((127 + (int)AT_P_SHIFT - min(code, (int)AT_CODE_CAP)) << 23);
+          // 2^(14 - code) as an fp32 exponent field: (127 + 14 - code) << 23, where the shift drops the
+          // 0x4B400000 of `bits` (its low 9 bits are zero).  Without the code output x is already held
+          // to the cap, beyond which the product would convert to an fp16 zero anyway.
+          const uint32_t capped = CODES ? min(bits, 0x4B400000u + (uint32_t)AT_CODE_CAP) : bits;
+          p[i] = __uint_as_float(((127u + (uint32_t)AT_P_SHIFT) << 23) - (capped << 23));
         }
         const __half2 ph = __floats2half2_rn(p[0], p[1]);
         pa[mt][nt >> 1][(nt & 1) * 2 + hi] = *reinterpret_cast<const uint32_t*>(&ph);
