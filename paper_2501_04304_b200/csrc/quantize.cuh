@@ -26,6 +26,7 @@ struct QuantArgs {
   uint8_t* Xq;
   int64_t M, ld;
   int C, K_pad, G, P, bits, rows_per_warp;
+  int rows_per_cta;        // a CTA takes this many consecutive rows per sweep (a multiple of rows_per_warp, at most one turn per warp)
   int dynamic, centred;
   const uint8_t* head;     // layout tables (see quant_head_bytes)
   const int32_t* row_group;
@@ -71,9 +72,14 @@ __global__ void __launch_bounds__(QA_THREADS, 4) quantize_act_kernel(const Quant
 
   const int vec_per_row = a.C >> 3;
   const float Lf = (float)((1 << a.bits) - 1);
-  const int64_t warps_total = (int64_t)gridDim.x * QA_WARPS;
-  for (int64_t row0 = ((int64_t)blockIdx.x * QA_WARPS + warp) * rpw; row0 < a.M; row0 += warps_total * rpw) {
-    const int rows = (int)min((int64_t)rpw, a.M - row0);
+  // A CTA takes rows_per_cta consecutive rows per sweep over the matrix, at most one turn per warp.  Small
+  // matrices are dealt out in one sweep with the same number of rows for every CTA (a kernel of one wave lasts
+  // as long as its busiest SM); large ones in sweeps of full CTAs.
+  for (int64_t base = (int64_t)blockIdx.x * a.rows_per_cta; base < a.M; base += (int64_t)gridDim.x * a.rows_per_cta) {
+    const int64_t cta_end = min(a.M, base + a.rows_per_cta);
+    const int64_t row0 = base + warp * rpw;
+    if (row0 >= cta_end) continue;  // the same answer in every lane of the warp
+    const int rows = (int)min((int64_t)rpw, cta_end - row0);
     // Row loads in batches of four 128-bit pieces per lane: every load of a batch is issued before
     // the first store, so the memory latency is paid once per batch and not once per piece.
     {
@@ -274,8 +280,24 @@ extern "C" dgq_status dgq_quantize_act(const dgq_groups* g, int timestep, int mo
     DGQ_CUDA_OK(cudaFuncSetAttribute(quantize_act_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
     if (dev < 64) attr_set[dev] = true;
   }
-  const int64_t n_ctas = (M + (int64_t)QA_WARPS * rpw - 1) / ((int64_t)QA_WARPS * rpw);
-  const int grid = (int)std::min<int64_t>(n_ctas, 148 * 8);
+  // Four CTAs fit on an SM.  A matrix that one wave of full CTAs can cover is dealt out evenly over 4 x SMs
+  // CTAs instead; a larger one goes to at most two waves of full CTAs that sweep over it.
+  static int sm_count[64] = {0};
+  if (dev >= 64 || sm_count[dev] == 0) {
+    int n = 0;
+    DGQ_CUDA_OK(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
+    if (n <= 0) return DGQ_ERR_CUDA;
+    if (dev < 64) sm_count[dev] = n;
+  }
+  const int64_t slots = 4 * (int64_t)(dev < 64 ? sm_count[dev] : 148);
+  const int64_t full = (int64_t)QA_WARPS * rpw;  // rows of a CTA whose warps all take one turn
+  int64_t rows_per_cta = full;
+  if (M <= slots * full) {
+    rows_per_cta = (M + slots - 1) / slots;
+    rows_per_cta = (rows_per_cta + rpw - 1) / rpw * rpw;
+  }
+  a.rows_per_cta = (int)rows_per_cta;
+  const int grid = (int)std::min<int64_t>((M + rows_per_cta - 1) / rows_per_cta, 2 * slots);
   DGQ_CUDA_OK(launch_pdl(quantize_act_kernel, dim3(grid), dim3(QA_THREADS), smem, (cudaStream_t)stream, a));
   g_launches += 1;
   DGQ_CUDA_OK(cudaGetLastError());
