@@ -14,6 +14,8 @@
 // HBM traffic: 2 B read + 1 B written per element (+ 8 B per (token, group) in dynamic mode).
 #pragma once
 
+#include <type_traits>
+
 #include "groups.cuh"
 
 namespace dgq {
@@ -183,24 +185,40 @@ __global__ void __launch_bounds__(QA_THREADS, 4) quantize_act_kernel(const Quant
         uint32_t w[4];
         if (abs(Z) <= (1 << 21)) {
           // Eq. 1 without conversion instructions, bit-identical to quantize_code for |Z| <= 2^21:
-          // t + 1.5 * 2^23 rounds t to the nearest-even integer (|t| < 2^22; a larger |t| ends at a
-          // clamp either way), subtracting (1.5 * 2^23 - Z) is exact and leaves rint(t) + Z, NaN
-          // falls to 0 in fmaxf, and after the clamps the code is the low byte of (q + 1.5 * 2^23).
+          // y = x * (1/s) + 1.5 * 2^23 carries rint(t) in its low mantissa bits (|t| < 2^22; a larger |t|
+          // ends at a clamp either way).  The lower clamp is taken on y (y >= 1.5 * 2^23 - Z means
+          // rint(t) + Z >= 0; NaN falls to the bound, hence to code 0, in fmaxf), then
+          // bits(y) - (0x4B400000 - Z) is the integer rint(t) + Z >= 0 and the upper clamp is an unsigned
+          // minimum.  The product and the sum are rounded separately (x * (1/s) + (-0) is the rounded
+          // product), two values per packed instruction.
           const float MAGIC = 12582912.0f;
-          const float mz = MAGIC - Zf, ms = MAGIC - (float)sub;
+          const float lowb = MAGIC - Zf;
+          const uint32_t Lu = (uint32_t)((1 << a.bits) - 1);
+          const unsigned long long inv2 = pack_f32x2(inv_s, inv_s), magic2 = pack_f32x2(MAGIC, MAGIC);
+          const unsigned long long nzero2 = pack_f32x2(-0.0f, -0.0f), one2 = pack_f32x2(1.0f, 1.0f);
+          const uint32_t off = 0x4B400000u - (uint32_t)Z;
+          auto codes16 = [&](auto centred_tag) {
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const float2 f0 = __half22float2(h[2 * q]), f1 = __half22float2(h[2 * q + 1]);
-            const float fv[4] = {f0.x, f0.y, f1.x, f1.y};
-            uint32_t b[4];
+            for (int q = 0; q < 4; ++q) {
+              uint32_t b[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              float v = __fsub_rn(__fadd_rn(__fmul_rn(fv[j], inv_s), MAGIC), mz);
-              v = fminf(fmaxf(v, 0.0f), Lf);
-              b[j] = __float_as_uint(__fadd_rn(v, ms));  // low byte = code - sub (two's complement)
+              for (int j = 0; j < 2; ++j) {
+                const float2 f = __half22float2(h[2 * q + j]);
+                const unsigned long long t2 = fma_f32x2(pack_f32x2(f.x, f.y), inv2, nzero2);
+                float y0, y1;
+                unpack_f32x2(fma_f32x2(t2, one2, magic2), y0, y1);
+                b[2 * j] = min(__float_as_uint(fmaxf(y0, lowb)) - off, Lu);
+                b[2 * j + 1] = min(__float_as_uint(fmaxf(y1, lowb)) - off, Lu);
+                if (decltype(centred_tag)::value) {  // low byte = code - Z (two's complement)
+                  b[2 * j] -= (uint32_t)sub;
+                  b[2 * j + 1] -= (uint32_t)sub;
+                }
+              }
+              w[q] = __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
             }
-            w[q] = __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
-          }
+          };
+          if (a.centred) codes16(std::true_type{});
+          else codes16(std::false_type{});
         } else {
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
