@@ -656,12 +656,20 @@ def run_micro(args):
         us = float(np.median(times[3:]))
         rec = {"case": name, "us": us, "gbs": algo_bytes / us / 1e3, "frac_hbm": algo_bytes / us / 1e3 / peaks["hbm"],
                "sets": len(fns), **extra}
+        t_hbm_us, t_tc_us = algo_bytes / peaks["hbm"] / 1e3, 0.0
         if algo_ops:
             rec["tops"] = algo_ops / us / 1e6
             if kind == "selfattn":      # fp16 operands: the measured bf16 peak is the denominator
                 rec["frac_f16_peak"] = rec["tops"] / peaks["bf16"]
+                t_tc_us = algo_ops / peaks["bf16"] / 1e6
             else:
                 rec["frac_int8_peak"] = rec["tops"] / (2 * peaks["bf16"])
+                t_tc_us = algo_ops / (2 * peaks["bf16"]) / 1e6
+        # the shape's own roofline: the slower of its algorithmic bytes at the measured copy bandwidth and its
+        # algorithmic operations at the measured (burst) tensor peak
+        rec["bound"] = "tensor" if t_tc_us > t_hbm_us else "hbm"
+        rec["roofline_us"] = max(t_tc_us, t_hbm_us)
+        rec["frac_roofline"] = rec["roofline_us"] / us
         assert b.device_status() == 0
         print(json.dumps(rec), flush=True)
         del sets, fns, graph
