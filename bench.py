@@ -383,10 +383,10 @@ def run_cuda(args):
     # at least K steps again, one graph per kind with an event in between, for the per-kernel split
     marks = []
     k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    kind_rounds = max(1, -(-args.steps // wl.KIND_STEPS))
-    kind_steps = kind_rounds * wl.KIND_STEPS
+    kind_replays = max(1, -(-args.steps // wl.KIND_STEPS))
+    kind_steps = kind_replays * wl.KIND_STEPS
     k0.record()
-    for _ in range(kind_rounds):
+    for _ in range(kind_replays):
         wl.replay_kinds(marks)
     k1.record()
     barrier()
