@@ -47,3 +47,17 @@ def test_noalloc_rejects_oversized_problem():
                                          C.c_int(300), C.c_int(1), C.c_int(1), C.c_int(4), C.c_int(40), C.c_int(8),
                                          C.c_int(0), None, C.c_void_p(O.data_ptr()), None, None, None)
     assert st == 4
+
+
+def test_noalloc_accepts_the_largest_problem():
+    """B * H = 256 heads and B * H * nq = 2^18 rows are the stated limits: the call must fit its scratch
+    (row statistics plus one partial maximum per block of query rows) and agree with the ordinary entry point."""
+    torch, b = gpu()
+    B, H, nq = 32, 8, 1024
+    Q, K, V = [to_dev(torch, x) for x in synth.attention_inputs(25, B, H, nq, 77, 40)]
+    O_ref, s_ref, _ = b.cross_attn_logq(Q, K, V, 8, want_scale=True)
+    O = torch.empty_like(Q)
+    s = torch.empty_like(s_ref)
+    b.cross_attn_logq_noalloc(Q, K, V, O, 8, scale_out=s)
+    assert b.device_status() == 0
+    assert torch.equal(s, s_ref) and torch.equal(O, O_ref)
