@@ -148,6 +148,8 @@ class Workload:
         Wc = torch.from_numpy(synth.conv_weights(SEED, 250, c["N"], c["c"])).to(dev)
         self.conv_weight = b.weight_prepare(self.conv_groups, Wc, 4, conv=self.conv_desc)
         self.conv_bias = torch.from_numpy(synth.bias(SEED, 350, c["N"])).to(dev)
+        self.conv_ws = torch.empty(b.linear_workspace_bytes(self.conv_groups, self.conv_weight, M), dtype=torch.uint8,
+                                   device=dev)   # the 4-bit conv weights are expanded into it by every call
         # host inputs (pinned) and device buffer sets
         self.host = {}
         for key, C in INPUT_C.items():
@@ -203,7 +205,7 @@ class Workload:
                 b.linear(self.groups[key], self.weights[name], s["codes"][key], mode=b.MODE_DYNAMIC_TOKEN,
                          dyn_scale=s["ds"][key], dyn_zp=s["dz"][key], bias=self.biases[name], out=s["out"][name])
             b.linear(self.conv_groups, self.conv_weight, s["conv_codes"], layout=b.CODES_S8_CENTRED,
-                     bias=self.conv_bias, out=s["conv_out"], conv=self.conv_desc)
+                     bias=self.conv_bias, out=s["conv_out"], conv=self.conv_desc, workspace=self.conv_ws)
         else:
             b.cross_attn_logq(s["in"]["Q"], s["in"]["K"], s["in"]["V"], ATT["bits"], out=s["attn_out"],
                               workspace=s["attn_ws"])
@@ -604,8 +606,10 @@ def run_micro(args):
                     w = b.weight_prepare(g, W, p["wbits"])
                     kreal, wb = C, p["wbits"]
                 bias = torch.from_numpy(synth.bias(SEED, 3, p["N"])).cuda()
+                ws_need = b.linear_workspace_bytes(g, w, M)      # 4-bit weights are expanded into it by every call
+                ws = torch.empty(ws_need, dtype=torch.uint8, device="cuda") if ws_need else None
                 fns = [lambda s=s: b.linear(g, w, s[1], mode=mode, layout=layout, dyn_scale=s[2], dyn_zp=s[3],
-                                            bias=bias, out=s[4], conv=conv) for s in sets]
+                                            bias=bias, out=s[4], conv=conv, workspace=ws) for s in sets]
                 algo_ops = 2.0 * M * p["N"] * kreal
                 algo_bytes = M * C + p["N"] * kreal * wb / 8 + 2.0 * M * p["N"]
             extra = {"K_pad": g.K_pad, "G": g.G}

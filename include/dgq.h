@@ -154,12 +154,21 @@ dgq_status dgq_weight_export(const dgq_weight* w, int8_t* wq, float* sw);
  * Y dev fp16 [M, N] with leading dimension ldy.  conv != NULL: 3x3 stride-1
  * zero-padded convolution of the NHWC code tensor as an implicit GEMM; needs
  * the S8_CENTRED layout, STATIC mode and channel-only grouping (R = 1).
- * Errors: INVALID_ARG, ALIGNMENT, NOT_CALIBRATED, UNSUPPORTED (K_pad * 255 * 127
- * would overflow int32; more column blocks of 128-160 outputs than the GPU has SMs;
- * conv shape outside the supported tiling), CUDA. */
+ * workspace: dev, 256-byte aligned, at least dgq_linear_workspace_bytes(); only
+ * 4-bit weights need one (a kernel in front of the GEMM expands them to bytes
+ * there, once per call instead of once per row tile; the bytes stay in L2).
+ * Contents undefined on entry and exit; calls that may overlap on the GPU need
+ * separate workspaces unless they use the same weight.  NULL / 0 for 8-bit
+ * weights.
+ * Errors: INVALID_ARG, ALIGNMENT, NOT_CALIBRATED, WORKSPACE, UNSUPPORTED (K_pad *
+ * 255 * 127 would overflow int32; more column blocks of 64-128 outputs than the
+ * GPU has SMs; conv shape outside the supported tiling), CUDA. */
 dgq_status dgq_linear(const dgq_groups* g, const dgq_weight* w, int timestep, int mode, int layout,
                       const void* Xq, const float* dyn_scale, const int32_t* dyn_zp, const void* bias,
-                      void* Y, int64_t M, int64_t ldy, const dgq_conv_desc* conv, void* stream);
+                      void* Y, int64_t M, int64_t ldy, const dgq_conv_desc* conv, void* workspace,
+                      size_t workspace_bytes, void* stream);
+/* Bytes of workspace dgq_linear needs for this weight and M rows (0 for 8-bit weights). */
+dgq_status dgq_linear_workspace_bytes(const dgq_groups* g, const dgq_weight* w, int64_t M, size_t* bytes);
 
 /* ---------------------------------------------------------------- cross-attention (Eq. 3, 8, 9)
  * Q dev fp16 [B, nq, H, d]; K, V dev fp16 [B, nk, H, d]; O dev fp16 [B, nq, H, d].

@@ -26,7 +26,7 @@ SCALE_PER_PROMPT, SCALE_PER_PROMPT_HEAD, SCALE_PER_CALL = 0, 1, 2
 EXPORTS = [
     "dgq_calibrate_groups", "dgq_groups_from_host", "dgq_groups_destroy", "dgq_groups_info",
     "dgq_groups_export", "dgq_quantize_act", "dgq_weight_prepare", "dgq_weight_from_codes",
-    "dgq_weight_destroy", "dgq_weight_export", "dgq_linear", "dgq_cross_attn_logq", "dgq_cross_attn_logq_qv", "dgq_self_attn_logq",
+    "dgq_weight_destroy", "dgq_weight_export", "dgq_linear", "dgq_linear_workspace_bytes", "dgq_cross_attn_logq", "dgq_cross_attn_logq_qv", "dgq_self_attn_logq",
     "dgq_cross_attn_workspace_bytes", "dgq_cross_attn_logq_noalloc", "dgq_device_status", "dgq_status_string", "dgq_launch_count",
 ]
 
@@ -238,14 +238,25 @@ def weight_from_codes(groups: Groups, wq, sw, w_bits=8, conv=None) -> Weight:
     return Weight(h, N, K)
 
 
+def linear_workspace_bytes(groups: Groups, weight: Weight, M: int) -> int:
+    n = C.c_size_t(0)
+    _check(lib().dgq_linear_workspace_bytes(groups.h, weight.h, C.c_int64(M), C.byref(n)), "dgq_linear_workspace_bytes")
+    return n.value
+
+
 def linear(groups: Groups, weight: Weight, Xq, timestep=0, mode=MODE_STATIC, layout=CODES_U8, dyn_scale=None,
-           dyn_zp=None, bias=None, out=None, conv=None, stream=None):
-    """dgq_linear.  Returns Y fp16 [M, N]."""
+           dyn_zp=None, bias=None, out=None, conv=None, workspace=None, stream=None):
+    """dgq_linear.  Returns Y fp16 [M, N].  `workspace` (uint8 CUDA tensor) is only needed for 4-bit
+    weights; when it is not given one of the size the library asks for is taken from torch."""
     M = Xq.shape[0]
     Y = out if out is not None else torch.empty((M, weight.N), dtype=torch.float16, device=Xq.device)
+    if workspace is None:
+        need = linear_workspace_bytes(groups, weight, M)
+        workspace = torch.empty(need, dtype=torch.uint8, device=Xq.device) if need else None
     st = lib().dgq_linear(groups.h, weight.h, C.c_int(timestep), C.c_int(mode), C.c_int(layout), _ptr(Xq),
                           _ptr(dyn_scale), _ptr(dyn_zp), _ptr(bias), _ptr(Y), C.c_int64(M), C.c_int64(Y.stride(0)),
-                          _conv(conv), _stream(stream))
+                          _conv(conv), _ptr(workspace), C.c_size_t(workspace.numel() if workspace is not None else 0),
+                          _stream(stream))
     _check(st, "dgq_linear")
     return Y
 

@@ -182,12 +182,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   }
 }
 
-// Bounded wait without a return value, for hot loops: after 2^21 parked polls (of at most a
+// Bounded wait without a return value, for hot loops: after `max_polls` (2^21) parked polls (of at most a
 // microsecond each) it records a time-out and raises `*abort_flag`; once the flag is up every wait
 // returns at its first failed poll.  The caller tests the flag at a coarser grain (once per tile)
 // and leaves through the kernel's common exit path; what it does in between only touches memory
 // the CTA owns.
-__device__ __forceinline__ void mbar_wait_lean(uint32_t bar_addr, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ void mbar_wait_lean(uint32_t bar_addr, uint32_t parity, volatile int* abort_flag,
+                                               uint32_t max_polls = 1u << 21) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
@@ -198,7 +199,7 @@ __device__ __forceinline__ void mbar_wait_lean(uint32_t bar_addr, uint32_t parit
       : "memory");
   if (ok) return;
   if (*abort_flag) return;
-  for (uint32_t spins = 0; spins < (1u << 21); ++spins) {
+  for (uint32_t spins = 0; spins < max_polls; ++spins) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
@@ -208,6 +209,40 @@ __device__ __forceinline__ void mbar_wait_lean(uint32_t bar_addr, uint32_t parit
         : "memory");
     if (ok) return;
     if ((spins & 31u) == 31u && *abort_flag) return;
+  }
+  *abort_flag = 1;
+  record_error(DGQ_ERR_TIMEOUT);
+}
+// Bounded wait for roles that may wait long while other warps of the CTA work: polls that answer at
+// once (test_wait) with a growing sleep in between (32 ns doubling to 256 ns), so that the waiting
+// warp takes almost no issue slots or shared-memory bandwidth from the working ones.  After 2^22
+// polls (about a second) it records a time-out and raises `*abort_flag`; once the flag is up every
+// wait returns at its first failed poll.
+__device__ __forceinline__ void mbar_wait_backoff(uint32_t bar_addr, uint32_t parity, volatile int* abort_flag,
+                                                  uint32_t max_polls = 1u << 22) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar_addr), "r"(parity)
+      : "memory");
+  if (ok) return;
+  if (*abort_flag) return;
+  uint32_t ns = 32;
+  for (uint32_t spins = 0; spins < max_polls; ++spins) {
+    asm volatile("nanosleep.u32 %0;" ::"r"(ns));
+    if (ns < 256) ns <<= 1;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar_addr), "r"(parity)
+        : "memory");
+    if (ok) return;
+    if ((spins & 63u) == 63u && *abort_flag) return;
   }
   *abort_flag = 1;
   record_error(DGQ_ERR_TIMEOUT);
@@ -224,6 +259,31 @@ __device__ __forceinline__ uint32_t mbar_try_addr(uint32_t bar_addr, uint32_t pa
       : "memory");
   return ok;
 }
+// The same without any waiting: try_wait may park the thread for a while when the phase is still
+// pending, test_wait answers at once.
+__device__ __forceinline__ uint32_t mbar_test_addr(uint32_t bar_addr, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar_addr), "r"(parity)
+      : "memory");
+  return ok;
+}
+// Read-only global loads that stay where they are written (a plain load may be moved next to its
+// first use, which would expose its latency there).
+__device__ __forceinline__ float ldg_f32_here(const float* p) {
+  float v;
+  asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ int ldg_s32_here(const int32_t* p) {
+  int v;
+  asm volatile("ld.global.nc.s32 %0, [%1];" : "=r"(v) : "l"(p));
+  return v;
+}
 // Register re-balancing between the warpgroups of a CTA (every warp of an aligned group of four
 // executes the same instruction).
 template <int REGS>
@@ -233,6 +293,15 @@ __device__ __forceinline__ void reg_alloc() {
 template <int REGS>
 __device__ __forceinline__ void reg_dealloc() {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS));
+}
+// True in exactly one lane of a converged warp.  A loop that the whole warp runs with uniform control
+// flow and whose tcgen05 instructions sit behind this test keeps its addresses and counters in the
+// uniform datapath, which makes the issuing path markedly shorter than a loop run by one lane of a
+// diverged warp.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+  return pred != 0;
 }
 __device__ __forceinline__ void mbar_arrive_addr(uint32_t bar_addr) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_addr) : "memory");
@@ -258,6 +327,18 @@ __device__ __forceinline__ void cvt_fma_f32x2(unsigned long long& y, unsigned lo
       : "r"(i0), "r"(i1), "l"(s2));
 }
 
+// Two int32 -> fp32 conversions straight into one 64-bit register pair (the operand form of the packed
+// fp32 instructions), so that no moves are needed to pair the results up.
+__device__ __forceinline__ unsigned long long cvt_s32x2_f32x2(uint32_t i0, uint32_t i1) {
+  unsigned long long r;
+  asm("{\n\t.reg .f32 f0, f1;\n\t"
+      "cvt.rn.f32.s32 f0, %1;\n\t"
+      "cvt.rn.f32.s32 f1, %2;\n\t"
+      "mov.b64 %0, {f0, f1};\n\t}"
+      : "=l"(r)
+      : "r"(i0), "r"(i1));
+  return r;
+}
 // d = a * b + c on two lanes
 __device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b,
                                                         unsigned long long c) {
@@ -368,6 +449,18 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
         "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+// 32 lanes x 32 consecutive 32-bit columns.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr)
       : "memory");
 }

@@ -32,6 +32,8 @@
 // the tap, out-of-image rows zero-filled by TMA (exact for zero-centred codes).
 #pragma once
 
+#include <type_traits>
+
 #include "weights.cuh"
 
 namespace dgq {
@@ -51,10 +53,10 @@ __host__ __device__ constexpr int gemm_threads(bool w4) { return (w4 ? 16 : 12) 
 // Registers per thread: the kernel starts with `gemm_regs_launch`, the epilogue warps then grow to
 // `gemm_regs_epi` with what the other warps give back (8 * epi + rest * other <= warps * launch).
 __host__ __device__ constexpr int gemm_regs_launch(bool w4) { return w4 ? 128 : 168; }
-__host__ __device__ constexpr int gemm_regs_epi(bool w4) { return w4 ? 200 : 208; }
-constexpr int GEMM_REGS_OTHER = 56;
-static_assert(8 * gemm_regs_epi(true) + 8 * GEMM_REGS_OTHER <= 16 * gemm_regs_launch(true), "register pool");
-static_assert(8 * gemm_regs_epi(false) + 4 * GEMM_REGS_OTHER <= 12 * gemm_regs_launch(false), "register pool");
+__host__ __device__ constexpr int gemm_regs_epi(bool w4) { return w4 ? 192 : 208; }
+__host__ __device__ constexpr int gemm_regs_other(bool w4) { return w4 ? 64 : 80; }
+static_assert(8 * gemm_regs_epi(true) + 8 * gemm_regs_other(true) <= 16 * gemm_regs_launch(true), "register pool");
+static_assert(8 * gemm_regs_epi(false) + 4 * gemm_regs_other(false) <= 12 * gemm_regs_launch(false), "register pool");
 constexpr int GEMM_MAX_ATOMS = 1024;           // 32768 reduction positions
 constexpr int GEMM_A_STAGE = GEMM_BM * 128;  // bytes
 constexpr int GEMM_SMEM_LIMIT = 227 * 1024;
@@ -204,7 +206,7 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   if (warp >= GEMM_EPI_WARPS) {
   // The warps that only move data or issue instructions hand most of their registers to the epilogue.
-  reg_dealloc<GEMM_REGS_OTHER>();
+  reg_dealloc<gemm_regs_other(W4)>();
   if (warp == GEMM_WARP_TMA) {
     // ------------------------------------------------------------ TMA producer
     // One lane runs the loop; the others go straight to the CTA's final barrier.
@@ -251,11 +253,13 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncwarp();
   } else if (warp == GEMM_WARP_MMA) {
     // ------------------------------------------------------------ MMA issuer
-    // One lane runs the loop.  Its dependent instruction chain per MMA is what bounds short groups,
-    // so everything that can be is precomputed (descriptor words, barrier addresses, the per-stage
-    // bit mask of atoms that end a group, running ring positions and parities) and the waits carry
-    // no warp votes.
-    if (lane == 0) {
+    // The whole warp runs the loop with uniform control flow; the tcgen05 instructions are issued by
+    // one elected lane.  What the issuing path costs per instruction, not the tensor core, bounds short
+    // groups: an MMA, a commit and a barrier poll each take tens to hundreds of cycles of this warp's
+    // time, whatever the tile width.  So a stage is straight-line code chosen by its pattern of group
+    // ends (no per-atom tests), everything that can be is precomputed (descriptor words, barrier
+    // addresses, running ring positions and parities).
+    {
       constexpr uint32_t A_HI = CONV ? smem_desc_hi(256, 6) : smem_desc_hi(1024, 2);
       constexpr uint32_t B_HI = smem_desc_hi(1024, 2);
       const uint32_t a_lo0 = smem_desc_lo(smem_u32(smA)), b_lo0 = smem_desc_lo(smem_u32(smB));
@@ -266,40 +270,54 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t full_phase = 0;   // parity of the slot's next "full" phase
       uint32_t ab = 0;           // accumulator of the next group
       uint32_t acc_phase = 1;    // parity to wait for on its "empty" barrier (fresh barriers pass)
+      // One stage of four atoms whose group ends are the bits of PAT; `need`: the first atom starts a group.
+      auto issue_stage = [&](auto pat_tag, bool need, uint32_t a_lo, uint32_t b_lo) {
+        constexpr int PAT = decltype(pat_tag)::value;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const bool starts = (j == 0) ? need : (((PAT >> (j > 0 ? j - 1 : 0)) & 1) != 0);
+          if (starts) {
+            mbar_wait_lean(acce0 + ab * 8u, acc_phase, abort_flag);
+            tc_fence_after();
+          }
+          if (elect_one()) {
+            mma_i8_lohi(tmem_base + ab * (uint32_t)BN, a_lo + (CONV ? j * 256 : j * 2), A_HI, b_lo + j * 2, B_HI, idesc,
+                        starts ? 0u : 1u);
+            if ((PAT >> j) & 1) mma_commit_addr(accf0 + ab * 8u);  // last atom of the group: hand the accumulator over
+          }
+          __syncwarp();
+          if ((PAT >> j) & 1) {
+            if (++ab == (uint32_t)NACC) {
+              ab = 0;
+              acc_phase ^= 1u;
+            }
+          }
+        }
+      };
       for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-        bool need_acc = true;  // the next atom starts a group: take the next accumulator first
-        uint32_t d_tmem = tmem_base;
+        bool need = true;      // every tile starts a group
         uint64_t ends = 0;     // bit i: atom (16 * 4) * word + i is the last of its group
         for (int ks = 0; ks < n_kstages; ++ks) {
           if ((ks & 15) == 0) ends = a.end_mask[ks >> 4];
-          const uint32_t end_bits = (uint32_t)(ends >> ((ks & 15) * 4)) & 0xFu;
+          uint32_t pat = (uint32_t)(ends >> ((ks & 15) * 4)) & 0xFu;
+          // A ragged last stage still issues four atoms (the missing ones multiply zero weights); the
+          // end of the last group moves to the last atom issued.
+          const int atoms_here = n_atoms - ks * 4;
+          if (atoms_here < 4) pat = (pat & ~(1u << (atoms_here - 1))) | 8u;
           mbar_wait_lean(full0 + s * 8u, full_phase, abort_flag);
           tc_fence_after();
-          const int atoms_here = min(4, n_atoms - ks * 4);
           const uint32_t a_lo = a_lo0 + s * (uint32_t)(GEMM_A_STAGE >> 4);
           const uint32_t b_lo = b_lo0 + s * (uint32_t)(Cfg::B_STAGE >> 4);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            if (j < atoms_here) {
-              if (need_acc) {
-                mbar_wait_lean(acce0 + ab * 8u, acc_phase, abort_flag);
-                tc_fence_after();
-                d_tmem = tmem_base + ab * (uint32_t)BN;
-              }
-              mma_i8_lohi(d_tmem, a_lo + (CONV ? j * 256 : j * 2), A_HI, b_lo + j * 2, B_HI, idesc,
-                          need_acc ? 0u : 1u);
-              need_acc = false;
-              if (end_bits & (1u << j)) {  // last atom of the group: hand the accumulator over right away
-                mma_commit_addr(accf0 + ab * 8u);
-                if (++ab == (uint32_t)NACC) {
-                  ab = 0;
-                  acc_phase ^= 1u;
-                }
-                need_acc = true;
-              }
-            }
+          switch (pat) {
+#define DGQ_STAGE_CASE(P) case P: issue_stage(std::integral_constant<int, P>{}, need, a_lo, b_lo); break;
+            DGQ_STAGE_CASE(0) DGQ_STAGE_CASE(1) DGQ_STAGE_CASE(2) DGQ_STAGE_CASE(3) DGQ_STAGE_CASE(4) DGQ_STAGE_CASE(5)
+            DGQ_STAGE_CASE(6) DGQ_STAGE_CASE(7) DGQ_STAGE_CASE(8) DGQ_STAGE_CASE(9) DGQ_STAGE_CASE(10) DGQ_STAGE_CASE(11)
+            DGQ_STAGE_CASE(12) DGQ_STAGE_CASE(13) DGQ_STAGE_CASE(14) DGQ_STAGE_CASE(15)
+#undef DGQ_STAGE_CASE
           }
-          mma_commit_addr(empty0 + s * 8u);  // stage reusable once these MMAs have read it
+          need = (pat & 8u) != 0;
+          if (elect_one()) mma_commit_addr(empty0 + s * 8u);  // stage reusable once these MMAs have read it
+          __syncwarp();
           if (++s == (uint32_t)STAGES) {
             s = 0;
             full_phase ^= 1u;
@@ -493,7 +511,7 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tmem_ld_wait();
         load_chunk(taddr + HC, rb1);
         // poll the next group's accumulator now, look at the answer after the arithmetic
-        const uint32_t next_ready = more ? mbar_try_addr(full0 + nab * 8u, npar) : 1u;
+        const uint32_t next_ready = more ? mbar_test_addr(full0 + nab * 8u, npar) : 1u;
 #pragma unroll
         for (int i = 0; i < HC / 2; ++i) cvt_fma_f32x2(y2[i], s2, rb0[2 * i], rb0[2 * i + 1]);
         if (!next_ready) mbar_wait_lean(full0 + nab * 8u, npar, abort_flag);
@@ -585,6 +603,20 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
 }
 
+// 4-bit weights -> bytes equal to 16 x the signed code (see pack_int4_words): one 16-byte packed piece
+// becomes 32 bytes.  Runs in front of the GEMM on the same stream when the caller provides a workspace;
+// the GEMM then reads the bytes like 8-bit weights (from L2) instead of expanding every stage of every
+// row tile again.
+__global__ void w4_expand_kernel(const uint4* __restrict__ packed, uint4* __restrict__ out, int64_t n_pieces) {
+  pdl_launch_dependents();
+  pdl_wait();  // the workspace may still be read by the GEMM of the layer before this one
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_pieces; i += (int64_t)gridDim.x * blockDim.x) {
+    const uint4 p4 = __ldg(packed + i);
+    out[2 * i] = make_uint4((p4.x << 4) & 0xF0F0F0F0u, p4.x & 0xF0F0F0F0u, (p4.y << 4) & 0xF0F0F0F0u, p4.y & 0xF0F0F0F0u);
+    out[2 * i + 1] = make_uint4((p4.z << 4) & 0xF0F0F0F0u, p4.z & 0xF0F0F0F0u, (p4.w << 4) & 0xF0F0F0F0u, p4.w & 0xF0F0F0F0u);
+  }
+}
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -654,8 +686,17 @@ static dgq_status launch_gemm_bn(bool w4, bool conv, const CUtensorMap& tmA, con
 
 extern "C" dgq_status dgq_linear(const dgq_groups* g, const dgq_weight* w, int timestep, int mode, int layout,
                                  const void* Xq, const float* dyn_scale, const int32_t* dyn_zp, const void* bias,
-                                 void* Y, int64_t M, int64_t ldy, const dgq_conv_desc* conv, void* stream) {
+                                 void* Y, int64_t M, int64_t ldy, const dgq_conv_desc* conv, void* workspace,
+                                 size_t workspace_bytes, void* stream) {
   using namespace dgq;
+  // 4-bit weights: with a workspace they are expanded once per call in front of the GEMM, without one
+  // the GEMM expands them itself, stage by stage
+  const size_t ws_need = w && w->w_bits == 4 ? (size_t)w->N_pad * (size_t)w->Kt : 0;
+  const bool expand_first = ws_need != 0 && workspace != nullptr;
+  if (expand_first) {
+    if (workspace_bytes < ws_need) return DGQ_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return DGQ_ERR_ALIGNMENT;
+  }
   if (!g || !w || !Xq || !Y || M <= 0) return DGQ_ERR_INVALID_ARG;
   if (mode != DGQ_MODE_STATIC && mode != DGQ_MODE_DYNAMIC_TOKEN) return DGQ_ERR_INVALID_ARG;
   if (layout != DGQ_CODES_U8 && layout != DGQ_CODES_S8_CENTRED) return DGQ_ERR_INVALID_ARG;
@@ -751,11 +792,12 @@ extern "C" dgq_status dgq_linear(const dgq_groups* g, const dgq_weight* w, int t
     const uint32_t box[2] = {128u, (uint32_t)GEMM_BM};
     if (!encode_map(&tmA, Xq, 2, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) return DGQ_ERR_CUDA;
   }
-  if (w->w_bits == 8) {
+  if (w->w_bits == 8 || expand_first) {
+    const void* wb = expand_first ? workspace : (const void*)w->d_w;
     const uint64_t dims[2] = {(uint64_t)w->Kt, (uint64_t)w->N_pad};
     const uint64_t strides[1] = {(uint64_t)w->Kt};
     const uint32_t box[2] = {128u, (uint32_t)BN};
-    if (!encode_map(&tmB, w->d_w, 2, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) return DGQ_ERR_CUDA;
+    if (!encode_map(&tmB, wb, 2, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B)) return DGQ_ERR_CUDA;
   }
   int dev = 0, n_sm = 148;
   DGQ_CUDA_OK(cudaGetDevice(&dev));
@@ -763,9 +805,22 @@ extern "C" dgq_status dgq_linear(const dgq_groups* g, const dgq_weight* w, int t
   // a multiple of the number of column blocks, so that every CTA keeps one column block
   if (a.n_tiles_n > n_sm) return DGQ_ERR_UNSUPPORTED;
   const int grid = std::min(a.n_tiles_m, n_sm / a.n_tiles_n) * a.n_tiles_n;
-  const bool w4 = (w->w_bits == 4);
+  const bool w4 = (w->w_bits == 4) && !expand_first;
   cudaStream_t st = (cudaStream_t)stream;
+  if (expand_first) {
+    const int64_t n_pieces = (int64_t)(ws_need / 32);  // 16 packed bytes each
+    const int blocks = (int)std::min<int64_t>((n_pieces + 255) / 256, (int64_t)n_sm * 8);
+    DGQ_CUDA_OK(launch_pdl(w4_expand_kernel, dim3(blocks), dim3(256), (size_t)0, st, (const uint4*)w->d_w, (uint4*)workspace,
+                           n_pieces));
+    g_launches += 1;
+  }
   if (BN == 160) return launch_gemm_bn<160>(w4, conv != nullptr, tmA, tmB, tmY, a, grid, st);
   if (BN == 64) return launch_gemm_bn<64>(w4, conv != nullptr, tmA, tmB, tmY, a, grid, st);
   return launch_gemm_bn<128>(w4, conv != nullptr, tmA, tmB, tmY, a, grid, st);
+}
+
+extern "C" dgq_status dgq_linear_workspace_bytes(const dgq_groups* g, const dgq_weight* w, int64_t M, size_t* bytes) {
+  if (!g || !w || !bytes || M <= 0) return DGQ_ERR_INVALID_ARG;
+  *bytes = w->w_bits == 4 ? (size_t)w->N_pad * (size_t)w->Kt : 0;
+  return DGQ_OK;
 }
