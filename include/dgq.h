@@ -234,7 +234,10 @@ dgq_status dgq_cross_attn_workspace_bytes(int B, int H, int nq, int nk, int d, s
  *     kernels can overlap on the GPU (different streams without an ordering
  *     between them) race on it:
  *     serialise them, or use dgq_cross_attn_logq with separate workspaces.
- * Errors: those of dgq_cross_attn_logq. */
+ * Errors: those of dgq_cross_attn_logq, checked first and in the same order; then
+ * DGQ_ERR_WORKSPACE for a problem beyond the limits above; DGQ_ERR_UNSUPPORTED when
+ * the current device's ordinal is 64 or more (the library remembers one address per
+ * device ordinal below that). */
 #define DGQ_NOALLOC_MAX_ROWS (1 << 18)
 #define DGQ_NOALLOC_MAX_HEADS 256
 #define DGQ_NOALLOC_SCRATCH_BYTES (4 * (DGQ_NOALLOC_MAX_ROWS / 128 + DGQ_NOALLOC_MAX_HEADS) + 8 * DGQ_NOALLOC_MAX_ROWS)
@@ -247,6 +250,11 @@ dgq_status dgq_cross_attn_logq_noalloc(const void* Q, const void* K, const void*
  * current device in *status (DGQ_OK, or the first error a kernel recorded),
  * then clears it. */
 dgq_status dgq_device_status(int* status);
+/* Diagnostic: enqueues a one-warp kernel whose only wait, on a barrier nobody arrives at, gives up
+ * after max_polls (1..65536) polls of at most a microsecond each, so that the time-out path of the
+ * bounded waits (status word, dgq_device_status, a usable device afterwards) can be exercised
+ * without making a wait of a working kernel run out.  Errors: INVALID_ARG, CUDA. */
+dgq_status dgq_selftest_wait_timeout(uint32_t max_polls, void* stream);
 const char* dgq_status_string(dgq_status s);
 /* Number of kernels the library has launched in this process (all devices). */
 uint64_t dgq_launch_count(void);

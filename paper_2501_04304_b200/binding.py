@@ -27,7 +27,7 @@ EXPORTS = [
     "dgq_calibrate_groups", "dgq_groups_from_host", "dgq_groups_destroy", "dgq_groups_info",
     "dgq_groups_export", "dgq_quantize_act", "dgq_weight_prepare", "dgq_weight_from_codes",
     "dgq_weight_destroy", "dgq_weight_export", "dgq_linear", "dgq_linear_workspace_bytes", "dgq_cross_attn_logq", "dgq_cross_attn_logq_qv", "dgq_self_attn_logq",
-    "dgq_cross_attn_workspace_bytes", "dgq_cross_attn_logq_noalloc", "dgq_device_status", "dgq_status_string", "dgq_launch_count",
+    "dgq_cross_attn_workspace_bytes", "dgq_cross_attn_logq_noalloc", "dgq_selftest_wait_timeout", "dgq_device_status", "dgq_status_string", "dgq_launch_count",
 ]
 
 
@@ -93,6 +93,11 @@ def device_status() -> int:
     v = C.c_int(0)
     _check(lib().dgq_device_status(C.byref(v)), "dgq_device_status")
     return v.value
+
+
+def selftest_wait_timeout(max_polls: int, stream=None):
+    """dgq_selftest_wait_timeout: a kernel whose only wait runs out after `max_polls` polls."""
+    _check(lib().dgq_selftest_wait_timeout(C.c_uint32(max_polls), _stream(stream)), "dgq_selftest_wait_timeout")
 
 
 class Groups:
@@ -246,11 +251,14 @@ def linear_workspace_bytes(groups: Groups, weight: Weight, M: int) -> int:
 
 def linear(groups: Groups, weight: Weight, Xq, timestep=0, mode=MODE_STATIC, layout=CODES_U8, dyn_scale=None,
            dyn_zp=None, bias=None, out=None, conv=None, workspace=None, stream=None):
-    """dgq_linear.  Returns Y fp16 [M, N].  `workspace` (uint8 CUDA tensor) is only needed for 4-bit
-    weights; when it is not given one of the size the library asks for is taken from torch."""
+    """dgq_linear.  Returns Y fp16 [M, N].  `workspace` (uint8 CUDA tensor) is only used for 4-bit
+    weights; when it is None one of the size the library asks for is taken from torch, when it is
+    False the call is made without one."""
     M = Xq.shape[0]
     Y = out if out is not None else torch.empty((M, weight.N), dtype=torch.float16, device=Xq.device)
-    if workspace is None:
+    if workspace is False:
+        workspace = None
+    elif workspace is None:
         need = linear_workspace_bytes(groups, weight, M)
         workspace = torch.empty(need, dtype=torch.uint8, device=Xq.device) if need else None
     st = lib().dgq_linear(groups.h, weight.h, C.c_int(timestep), C.c_int(mode), C.c_int(layout), _ptr(Xq),

@@ -527,10 +527,9 @@ extern "C" dgq_status dgq_cross_attn_workspace_bytes(int B, int H, int nq, int n
 }
 
 namespace dgq {
-static dgq_status attn_run(const void* Q, const void* K, const void* V, int B, int H, int nq, int nk, int d,
-                           int score_bits, int scale_gran, const float* fixed_scale, int v_bits, void* O,
-                           float* scale_out, uint8_t* codes_out, void* workspace, size_t workspace_bytes,
-                           void* stream) {
+// The argument checks every cross-attention entry point makes first, in this order.
+static dgq_status attn_check_args(const void* Q, const void* K, const void* V, int B, int H, int nq, int nk, int d,
+                                  int score_bits, int scale_gran, int v_bits, const void* O) {
   if (!Q || !K || !V || !O || B <= 0 || H <= 0 || nq <= 0 || d <= 0) return DGQ_ERR_INVALID_ARG;
   if (v_bits != 0 && (v_bits < 2 || v_bits > 8)) return DGQ_ERR_INVALID_ARG;
   if (nk < 2) return DGQ_ERR_INVALID_ARG;
@@ -538,6 +537,15 @@ static dgq_status attn_run(const void* Q, const void* K, const void* V, int B, i
   if (scale_gran < DGQ_SCALE_PER_PROMPT || scale_gran > DGQ_SCALE_PER_CALL) return DGQ_ERR_INVALID_ARG;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return DGQ_ERR_ALIGNMENT;
   if (nk > 128 || (d != 40 && d != 64 && d != 80 && d != 128 && d != 160)) return DGQ_ERR_UNSUPPORTED;
+  return DGQ_OK;
+}
+
+static dgq_status attn_run(const void* Q, const void* K, const void* V, int B, int H, int nq, int nk, int d,
+                           int score_bits, int scale_gran, const float* fixed_scale, int v_bits, void* O,
+                           float* scale_out, uint8_t* codes_out, void* workspace, size_t workspace_bytes,
+                           void* stream) {
+  dgq_status chk = attn_check_args(Q, K, V, B, H, nq, nk, d, score_bits, scale_gran, v_bits, O);
+  if (chk != DGQ_OK) return chk;
   size_t need = 0;
   dgq_cross_attn_workspace_bytes(B, H, nq, nk, d, &need);
   if (!workspace || workspace_bytes < need) return DGQ_ERR_WORKSPACE;

@@ -27,7 +27,9 @@ extern "C" dgq_status dgq_cross_attn_logq_noalloc(const void* Q, const void* K, 
                                                   int nk, int d, int score_bits, int scale_gran,
                                                   const float* fixed_scale, void* O, float* scale_out,
                                                   uint8_t* codes_out, void* stream) {
-  if (B <= 0 || H <= 0 || nq <= 0) return DGQ_ERR_INVALID_ARG;
+  // the ordinary argument errors come first, then the limits of the built-in scratch
+  dgq_status chk = dgq::attn_check_args(Q, K, V, B, H, nq, nk, d, score_bits, scale_gran, 0, O);
+  if (chk != DGQ_OK) return chk;
   if ((int64_t)B * H > DGQ_NOALLOC_MAX_HEADS || (int64_t)B * H * nq > DGQ_NOALLOC_MAX_ROWS)
     return DGQ_ERR_WORKSPACE;  // larger than the built-in scratch: use dgq_cross_attn_logq
   int dev = 0;
@@ -47,6 +49,30 @@ extern "C" dgq_status dgq_cross_attn_logq_noalloc(const void* Q, const void* K, 
   // that the second one reads, so stale contents from an earlier call are harmless.
   return dgq_cross_attn_logq(Q, K, V, B, H, nq, nk, d, score_bits, scale_gran, fixed_scale, O, scale_out,
                              codes_out, scratch, (size_t)DGQ_NOALLOC_SCRATCH_BYTES, stream);
+}
+
+namespace dgq {
+// One warp waits, with the caller's poll limit, on a barrier that nobody arrives at: the bounded wait
+// gives up, records DGQ_ERR_TIMEOUT and the kernel ends normally.
+__global__ void selftest_wait_kernel(uint32_t max_polls) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    fence_barrier_init();
+  }
+  __syncthreads();
+  mbar_wait_lean(smem_u32(&bar), 0u, &abort_flag, max_polls);
+}
+}  // namespace dgq
+
+extern "C" dgq_status dgq_selftest_wait_timeout(uint32_t max_polls, void* stream) {
+  if (max_polls == 0 || max_polls > (1u << 16)) return DGQ_ERR_INVALID_ARG;
+  dgq::selftest_wait_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(max_polls);
+  dgq::g_launches += 1;
+  DGQ_CUDA_OK(cudaGetLastError());
+  return DGQ_OK;
 }
 
 extern "C" dgq_status dgq_device_status(int* status) {

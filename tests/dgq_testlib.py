@@ -1,4 +1,6 @@
 """Helpers shared by the GPU parity tests: run the oracle and the CUDA library on the same seeded inputs."""
+import os
+
 import numpy as np
 import pytest
 
@@ -56,3 +58,32 @@ def check_output(Y_gpu, Y_ref, rel=1e-3):
     bound = rel * np.max(np.abs(Y_ref))
     assert err <= bound, f"max|delta| {err:.3e} > {rel} * max|ref| = {bound:.3e}"
     return err / np.max(np.abs(Y_ref))
+
+
+CODE_FRAC = 1e-4   # log2 codes may differ from the oracle's by one level on at most this fraction of the entries
+
+
+def check_codes(c, codes_ref):
+    """Integer codes against the oracle's: never more than one level apart, and different on at most
+    CODE_FRAC of the entries (rounded up to a whole entry, so the smallest cases tolerate one).  With
+    DGQ_FLIP_REPORT set to a file name the measured counts are appended there.  Returns the absolute
+    difference array."""
+    diff = np.abs(np.asarray(c, dtype=np.int64) - np.asarray(codes_ref, dtype=np.int64))
+    assert diff.max() <= 1, "a code differs by more than one level"
+    n_flips = int((diff != 0).sum())
+    path = os.environ.get("DGQ_FLIP_REPORT")
+    if path:
+        with open(path, "a") as fh:
+            fh.write(f"{os.environ.get('PYTEST_CURRENT_TEST', '')} entries {diff.size} flips {n_flips}\n")
+    allowed = int(np.ceil(CODE_FRAC * diff.size))
+    assert n_flips <= allowed, f"{n_flips} of {diff.size} codes differ (allowed {allowed})"
+    return diff
+
+
+def flipped_output_bound(diff, c, codes_ref, s, V_rest):
+    """How far a row's output may move when some of its codes sit one level off: an entry whose code is c
+    instead of c +- 1 changes its weight s 2^-code by s 2^-max(codes), times |V_j| per feature.
+    diff, c, codes_ref [B, H, nq, n]; s broadcastable to them; V_rest [B, n, H, d] -> bound [B, nq, H, d]."""
+    w = np.where(diff != 0, np.ldexp(np.broadcast_to(s, diff.shape).astype(np.float64),
+                                     -np.maximum(c, codes_ref).astype(np.int64)), 0.0)
+    return np.einsum("bhqk,bkhd->bqhd", w, np.abs(np.asarray(V_rest, dtype=np.float64)))

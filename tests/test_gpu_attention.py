@@ -4,12 +4,12 @@ import pytest
 
 from oracle import attention as oa
 from paper_2501_04304_b200 import synth
-from dgq_testlib import gpu, to_dev, check_output
+from dgq_testlib import gpu, to_dev, check_output, check_codes, flipped_output_bound
 
 pytestmark = pytest.mark.gpu
 
 
-def _compare(torch, b, Q, K, V, bits, gran=0, fixed=None, code_frac=1e-4, out_rel=1e-3, v_bits=None):
+def _compare(torch, b, Q, K, V, bits, gran=0, fixed=None, out_rel=1e-3, v_bits=None):
     O_ref, codes_ref, s_ref, A = oa.cross_attn_logq(Q, K, V, bits, gran, fixed, v_bits=v_bits)
     fx = to_dev(torch, np.asarray(fixed, np.float32)) if fixed is not None else None
     O, scale, codes = b.cross_attn_logq(to_dev(torch, Q), to_dev(torch, K), to_dev(torch, V), bits, gran, fx,
@@ -20,18 +20,16 @@ def _compare(torch, b, Q, K, V, bits, gran=0, fixed=None, code_frac=1e-4, out_re
     s_gpu = scale.cpu().numpy().astype(np.float64)
     assert np.allclose(s_gpu, s_ref.ravel(), rtol=2e-5, atol=0)
     c = codes.cpu().numpy().astype(np.int64)
-    diff = np.abs(c - codes_ref)
-    assert diff.max() <= 1, "a code differs by more than one level"
-    frac = (diff != 0).mean()
-    assert frac <= code_frac, f"{frac:.2e} of the codes differ"
-    # A score that sits on a rounding boundary may take either neighbouring level (softmax rounding);
-    # one flipped level moves the output by up to half that score times |V|.  Rows whose codes all agree
-    # are held to the oracle's output; the others to Eq. 9 evaluated with the codes the kernel chose.
-    O_alt = oa.split_product(A, c, s_ref, V)
-    flipped = (diff != 0).any(axis=-1).transpose(0, 2, 1)          # [B, nq, H]
-    assert np.array_equal(O_alt[~flipped], O_ref[~flipped])
-    check_output(O, O_alt, out_rel)
-    return frac
+    diff = check_codes(c, codes_ref)
+    # A score that sits on a rounding boundary may take either neighbouring level (softmax rounding).
+    # The output is held to the oracle's own output, every row, with the allowance that the row's
+    # flipped codes (if any) explain and nothing more ...
+    Og = O.float().cpu().numpy().astype(np.float64)
+    bound = out_rel * np.max(np.abs(O_ref)) + flipped_output_bound(diff, c, codes_ref, s_ref, V[:, 1:])
+    assert np.all(np.abs(Og - O_ref) <= bound), f"max excess {np.max(np.abs(Og - O_ref) - bound):.3e}"
+    # ... and, tighter, to Eq. 9 evaluated with the codes the kernel chose.
+    check_output(O, oa.split_product(A, c, s_ref, V), out_rel)
+    return int((diff != 0).sum())
 
 
 @pytest.mark.parametrize("bits", [8, 4])
@@ -52,20 +50,20 @@ def test_small_config3_like(bits):
 def test_shapes(B, H, nq, nk, d):
     torch, b = gpu()
     Q, K, V = synth.attention_inputs(4, B, H, nq, nk, d, ctx_dim=64)
-    _compare(torch, b, Q, K, V, 8, code_frac=5e-4)
+    _compare(torch, b, Q, K, V, 8)
 
 
 @pytest.mark.parametrize("gran", [0, 1, 2])
 def test_scale_granularity(gran):
     torch, b = gpu()
     Q, K, V = synth.attention_inputs(5, 3, 4, 200, 77, 40, ctx_dim=64)
-    _compare(torch, b, Q, K, V, 6, gran=gran, code_frac=5e-4)
+    _compare(torch, b, Q, K, V, 6, gran=gran)
 
 
 def test_fixed_scale_variant():
     torch, b = gpu()
     Q, K, V = synth.attention_inputs(6, 2, 2, 128, 77, 40, ctx_dim=64)
-    _compare(torch, b, Q, K, V, 8, fixed=[0.05, 0.01], code_frac=5e-4)
+    _compare(torch, b, Q, K, V, 8, fixed=[0.05, 0.01])
 
 
 def test_wide_logits_saturate_four_bits():
@@ -77,7 +75,7 @@ def test_wide_logits_saturate_four_bits():
     for bits in (4, 8):
         O_ref, codes_ref, _, _ = oa.cross_attn_logq(Q, K, V, bits)
         assert codes_ref.max() == (15 if bits == 4 else codes_ref.max()) and codes_ref.max() >= 15
-        _compare(torch, b, Q, K, V, bits, code_frac=1e-3)
+        _compare(torch, b, Q, K, V, bits)
 
 
 def test_uniform_and_one_hot_scores():
@@ -96,8 +94,8 @@ def test_uniform_and_one_hot_scores():
     K1[:, 0, :, -1] = np.float16(60.0 * np.sqrt(40))      # the <start> column gets e^60 times the others' weight
     O_ref, codes_ref, _, _ = oa.cross_attn_logq(Q, K1, V, 4)
     assert np.allclose(O_ref, V[:, :1].astype(np.float64), rtol=0, atol=1e-6)
-    _compare(torch, b, Q, K1, V, 4, code_frac=1e-3)
-    _compare(torch, b, Q, K1, V, 8, code_frac=1e-3)
+    _compare(torch, b, Q, K1, V, 4)
+    _compare(torch, b, Q, K1, V, 8)
 
 
 def test_argument_errors():
@@ -125,7 +123,7 @@ def test_quantized_value_operand(v_bits):
 def test_quantized_value_operand_shapes(B, H, nq, nk, d):
     torch, b = gpu()
     Q, K, V = synth.attention_inputs(9, B, H, nq, nk, d, ctx_dim=64)
-    _compare(torch, b, Q, K, V, 8, code_frac=5e-4, v_bits=8)
+    _compare(torch, b, Q, K, V, 8, v_bits=8)
 
 
 def test_quantized_value_operand_rejects_bad_bits():

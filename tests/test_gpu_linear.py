@@ -130,3 +130,72 @@ def test_linear_argument_errors():
     with pytest.raises(b.DgqError) as e:          # output not 16-byte aligned
         b.linear(g, w, Xq, out=Y)
     assert e.value.status == 2
+
+
+@pytest.mark.parametrize("w_bits", [8, 4])
+def test_objects_rebuilt_from_exports_give_identical_results(w_bits):
+    """dgq_groups_export -> dgq_groups_from_host and dgq_weight_export -> dgq_weight_from_codes: the rebuilt
+    grouping has the same layout and tables, the rebuilt weight the same codes, and the layer output is bit for
+    bit the same (static grid with pixel and channel groups)."""
+    torch, b = gpu()
+    P, C, N, K = 256, 320, 320, 4
+    Xcal, X, W, bias, gr = layer_case(14, 2, P, C, N, K, 8, oc.DIM_BOTH)
+    g = b.calibrate_groups(to_dev(torch, Xcal), P, 8, K, b.DIM_BOTH)
+    ex = g.export()
+    g2 = b.groups_from_host(C, P, 8, ex["col_group"], ex["row_group"], ex["scale"], ex["zp"])
+    ex2 = g2.export()
+    assert (g2.G, g2.R, g2.T, g2.K_pad, g2.bits) == (g.G, g.R, g.T, g.K_pad, g.bits)
+    for k in ("perm", "col_group", "group_off", "row_group", "scale", "zp"):
+        assert np.array_equal(ex[k], ex2[k]), k
+    w = b.weight_prepare(g, to_dev(torch, W), w_bits)
+    wq, sw = w.export()
+    w2 = b.weight_from_codes(g2, wq, sw, w_bits)
+    wq2, sw2 = w2.export()
+    assert np.array_equal(wq, wq2) and np.array_equal(sw, sw2)
+    Xd, bd = to_dev(torch, X), to_dev(torch, bias)
+    Xq, _, _ = b.quantize_act(g, Xd)
+    Xq2, _, _ = b.quantize_act(g2, Xd)
+    assert torch.equal(Xq, Xq2)
+    Y = b.linear(g, w, Xq, bias=bd)
+    Y2 = b.linear(g2, w2, Xq2, bias=bd)
+    assert torch.equal(Y, Y2)
+    codes, s_rows, z_rows = ol.quantize_static(X, gr, 0)
+    check_output(Y2, ol.group_linear(codes, s_rows, z_rows, gr.col_group, *ol.weight_rtn(W, w_bits), bias), REL)
+    assert b.device_status() == 0
+
+
+def test_four_bit_weights_with_and_without_workspace():
+    """4-bit weights take two routes: expanded once per call into the caller's workspace in front of the GEMM, or,
+    without a workspace, expanded stage by stage inside it.  Same integers either way: identical outputs."""
+    torch, b = gpu()
+    M, C, N, K = 1000, 640, 640, 8
+    Xcal, X, W, bias, gr = layer_case(15, 1, M, C, N, K, 8, oc.DIM_CHANNEL)
+    g = b.calibrate_groups(to_dev(torch, Xcal), M, 8, K, b.DIM_CHANNEL)
+    w = b.weight_prepare(g, to_dev(torch, W), 4)
+    need = b.linear_workspace_bytes(g, w, M)
+    assert need > 0
+    Xq, ds, dz = b.quantize_act(g, to_dev(torch, X), mode=b.MODE_DYNAMIC_TOKEN)
+    kw = dict(mode=b.MODE_DYNAMIC_TOKEN, dyn_scale=ds, dyn_zp=dz, bias=to_dev(torch, bias))
+    Y_ws = b.linear(g, w, Xq, workspace=torch.empty(need, dtype=torch.uint8, device="cuda"), **kw)
+    Y_in = b.linear(g, w, Xq, workspace=False, **kw)
+    assert torch.equal(Y_ws, Y_in)
+    with pytest.raises(b.DgqError) as e:          # a workspace that is too small is refused
+        b.linear(g, w, Xq, workspace=torch.empty(need // 2, dtype=torch.uint8, device="cuda"), **kw)
+    assert e.value.status == 4
+    codes, s_rows, z_rows = ol.quantize_dynamic_token(X, gr.col_group, gr.G, gr.bits)
+    check_output(Y_ws, ol.group_linear(codes, s_rows, z_rows, gr.col_group, *ol.weight_rtn(W, 4), bias), REL)
+    assert b.device_status() == 0
+
+
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_device_usable():
+    """Every device-side wait is bounded.  The library's self-test kernel waits, with a short limit, on a barrier
+    nobody arrives at: the status word reads DGQ_ERR_TIMEOUT once, is clear afterwards, and a layer call right
+    after it gives the right result."""
+    torch, b = gpu()
+    assert b.device_status() == 0
+    b.selftest_wait_timeout(2000)
+    assert b.device_status() == 6
+    assert b.device_status() == 0
+    Xcal, X, W, bias, gr = layer_case(16, 1, 256, 320, 320, 4, 8, oc.DIM_CHANNEL)
+    g = b.calibrate_groups(to_dev(torch, Xcal), 256, 8, 4, b.DIM_CHANNEL)
+    _run_linear(torch, b, X, W, bias, gr, g, "dynamic", 8)

@@ -4,6 +4,7 @@ import pytest
 
 from oracle import calibration as oc
 from oracle import linear as ol
+from oracle.quantizers import quantize_canonical_f32
 from paper_2501_04304_b200 import synth
 from dgq_testlib import gpu, to_dev, unpermute_codes, oracle_grouping_matches, layer_case
 
@@ -147,3 +148,45 @@ def test_dynamic_token_degenerate_rows():
     big = np.clip(Yref[~ordinary], -65504.0, 65504.0)
     got = np.nan_to_num(Yg[~ordinary], posinf=65504.0, neginf=-65504.0)
     assert np.max(np.abs(got - big)) <= 1e-3 * np.max(np.abs(big))
+
+
+def test_nonfinite_inputs_static_both_code_paths():
+    """NaN -> code 0, +inf -> the last code, -inf -> 0 (the fmax / fmin semantics of the fixed fp32 order), through
+    the conversion-free code path (|Z| <= 2^21) and the canonical one (a zero-point far outside it), with tables
+    handed over from the host.  Ordinary values around the specials must be unaffected."""
+    torch, b = gpu()
+    C, P, bits = 64, 16, 8
+    col_group = (np.arange(C) // 16).astype(np.int32)                # 4 groups of 16 channels
+    scale = np.array([[[0.05, 1e-6, 0.01, 2.0]]], np.float32)        # [T=1, R=1, G=4]
+    zp = np.array([[[100, 5_000_000, -3_000_000, 255]]], np.int32)   # groups 1 and 2 are beyond 2^21
+    g = b.groups_from_host(C, P, bits, col_group, np.zeros(P, np.int32), scale, zp)
+    assert (g.G, g.R, g.T) == (4, 1, 1)
+    rng = np.random.default_rng(5)
+    X = rng.normal(0, 3, (48, C)).astype(np.float16)
+    X[:, 16:32] = (5.0 + rng.normal(0, 1e-4, (48, 16))).astype(np.float16)      # near -Z s of group 1
+    X[:, 32:48] = (-30000.0 + rng.normal(0, 50, (48, 16))).astype(np.float16)   # near -Z s of group 2
+    for r, v in enumerate([np.nan, np.inf, -np.inf]):
+        X[r::8, r::5] = v                                            # specials in every group and chunk position
+    inv = (np.float32(1.0) / scale[0, 0]).astype(np.float32)
+    ref = quantize_canonical_f32(X, inv[col_group][None, :], zp[0, 0][col_group][None, :], bits)
+    assert set(np.unique(ref[np.isnan(X.astype(np.float32))])) == {0}
+    assert set(np.unique(ref[np.isposinf(X.astype(np.float32))])) == {255}
+    assert set(np.unique(ref[np.isneginf(X.astype(np.float32))])) == {0}
+    Xq, _, _ = b.quantize_act(g, to_dev(torch, X))
+    assert np.array_equal(unpermute_codes(Xq, g.export()["perm"], C), ref)
+    assert b.device_status() == 0
+
+
+def test_static_grid_at_8192_rows():
+    """Both outlier types at the benchmark's size: 2 x 4096 tokens x 320 channels, a grid of pixel groups x
+    channel groups; every code of the whole matrix against the oracle."""
+    torch, b = gpu()
+    P, C, K = 4096, 320, 4
+    Xcal, X, W, bias, gr = layer_case(13, 2, P, C, 8, K, 8, oc.DIM_BOTH)
+    g = b.calibrate_groups(to_dev(torch, Xcal), P, 8, K, b.DIM_BOTH)
+    assert g.R > 1 and g.G > 1
+    oracle_grouping_matches(gr, g.export())
+    ref, _, _ = ol.quantize_static(X, gr, 0)
+    Xq, _, _ = b.quantize_act(g, to_dev(torch, X))
+    assert np.array_equal(unpermute_codes(Xq, g.export()["perm"], C), ref)
+    assert b.device_status() == 0

@@ -24,7 +24,15 @@ def test_noalloc_matches_workspace_entry_point_twice():
         O = torch.empty_like(Q)
         s = torch.empty_like(s_ref)
         c = torch.empty_like(c_ref)
+        if call == 1:
+            # the entry point itself takes no device memory: neither the driver's free-memory figure nor
+            # torch's allocator moves across the call (every buffer above was made before it)
+            torch.cuda.synchronize()
+            free0, alloc0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
         b.cross_attn_logq_noalloc(Q, K, V, O, bits, scale_out=s, codes_out=c)
+        if call == 1:
+            torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info()[0] == free0 and torch.cuda.memory_allocated() == alloc0
         assert b.device_status() == 0
         ref = O_ref.float().cpu().numpy()
         got = O.float().cpu().numpy()
@@ -47,6 +55,16 @@ def test_noalloc_rejects_oversized_problem():
                                          C.c_int(300), C.c_int(1), C.c_int(1), C.c_int(4), C.c_int(40), C.c_int(8),
                                          C.c_int(0), None, C.c_void_p(O.data_ptr()), None, None, None)
     assert st == 4
+    # few heads but too many rows for the row statistics
+    st = lib.dgq_cross_attn_logq_noalloc(C.c_void_p(Q.data_ptr()), C.c_void_p(K.data_ptr()), C.c_void_p(V.data_ptr()),
+                                         C.c_int(1), C.c_int(8), C.c_int(40000), C.c_int(4), C.c_int(40), C.c_int(8),
+                                         C.c_int(0), None, C.c_void_p(O.data_ptr()), None, None, None)
+    assert st == 4
+    # an ordinary argument error on an oversized problem is reported as what it is (nk < 2: invalid argument)
+    st = lib.dgq_cross_attn_logq_noalloc(C.c_void_p(Q.data_ptr()), C.c_void_p(K.data_ptr()), C.c_void_p(V.data_ptr()),
+                                         C.c_int(64), C.c_int(8), C.c_int(4096), C.c_int(1), C.c_int(40), C.c_int(8),
+                                         C.c_int(0), None, C.c_void_p(O.data_ptr()), None, None, None)
+    assert st == 1
 
 
 def test_noalloc_accepts_the_largest_problem():
