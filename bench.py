@@ -73,6 +73,36 @@ def measured_peaks():
     return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
 
 
+# Plain-ALU bound of the per-group epilogue: every accumulator element of every channel group takes one
+# int32 -> fp32 conversion, which the SM issues at 16 per clock and sub-partition (64 per SM).
+CVT_PER_CLK_SM = 64
+
+
+def alu_peak_gelems(n_sm=148, sm_mhz=1965.0):
+    """Conversions per second of the whole GPU, in 1e9 elements / s."""
+    return CVT_PER_CLK_SM * n_sm * sm_mhz * 1e6 / 1e9
+
+
+def gemm_launch_rooflines(peaks, int8_peak_tops, n_sm, sm_mhz):
+    """Per GEMM launch of the step: (ops, bytes, group elements) and its own roofline time in us: the slowest of
+    tensor, HBM and epilogue-conversion time."""
+    out = []
+    alu = alu_peak_gelems(n_sm, sm_mhz)
+    for name, N, K, key in LINEARS:
+        ops, byts, el = 2.0 * M * N * K, M * K + N * K + 2.0 * M * N, float(M) * N * 8
+        out.append((name, ops, byts, el))
+    c = CONV
+    Mc = c["n"] * c["h"] * c["w"]
+    out.append(("conv", 2.0 * Mc * c["N"] * 9 * c["c"], Mc * c["c"] + c["N"] * 9 * c["c"] / 2 + 2.0 * Mc * c["N"],
+                float(Mc) * c["N"] * 16))
+    res = []
+    for name, ops, byts, el in out:
+        t = {"tensor": ops / int8_peak_tops / 1e6, "hbm": byts / peaks["hbm"] / 1e3, "alu": el / alu / 1e3}
+        bound = max(t, key=t.get)
+        res.append({"launch": name, "bound": bound, "roofline_us": t[bound], "t_us": t})
+    return res
+
+
 class ClockSampler(threading.Thread):
     """Samples SM clocks and throttle reasons with ONE long-running `nvidia-smi -lms` child, started before
     the warm-up so that no process is spawned while a timed region runs; `mark()` opens the window whose
@@ -371,7 +401,16 @@ def run_cuda(args):
     for _ in range(2):
         wl.replay_kinds()
     barrier()
+    # A step lasts a fraction of a millisecond: the K timed steps are preceded by about a second of untimed
+    # replays of the same graphs, so that the clock record below has tens of samples taken under this load.
     sampler.mark()
+    t_load = time.monotonic()
+    i_load = 0
+    while time.monotonic() - t_load < 1.0:
+        for _ in range(200):
+            wl.replay_whole_step(i_load)
+            i_load += 1
+        torch.cuda.synchronize()
     # timed region: K whole steps, one graph replay each
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
@@ -420,6 +459,23 @@ def run_cuda(args):
     attn_ms = sum(kind_ms["attention"]) / kind_steps
     quant_ms = sum(kind_ms["quantize"]) / kind_steps
     quant_bytes = 3.0 * (M * sum(INPUT_C.values()) + M * CONV["c"])
+    props = torch.cuda.get_device_properties(local)
+    sm_mhz = clocks.get("sm_max_mhz") or 1965.0
+    int8_burst = 2.0 * peaks["bf16"]
+    launches_rf = gemm_launch_rooflines(peaks, int8_peak, props.multi_processor_count, sm_mhz)
+    # the resource that binds most of the step's GEMM time, and the step's GEMM roofline = sum of the launches' own
+    sums = {k: sum(l["t_us"][k] for l in launches_rf) for k in ("tensor", "hbm", "alu")}
+    bound = max(sums, key=sums.get)
+    own_us = sum(l["roofline_us"] for l in launches_rf)
+    gemm_elems = sum(float(M) * N * 8 for _, N, _, _ in LINEARS) + float(M) * CONV["N"] * 16
+    gemm_bytes = sum(M * K + N * K + 2.0 * M * N for _, N, K, _ in LINEARS) + M * CONV["c"] + CONV["N"] * 9 * CONV["c"] / 2 \
+        + 2.0 * M * CONV["N"]
+    if bound == "tensor":
+        ach, peak, unit = gemm_tops, int8_peak, "TOP/s"
+    elif bound == "hbm":
+        ach, peak, unit = gemm_bytes / (gemm_ms * 1e-3) / 1e9, peaks["hbm"], "GB/s"
+    else:
+        ach, peak, unit = gemm_elems / (gemm_ms * 1e-3) / 1e9, alu_peak_gelems(props.multi_processor_count, sm_mhz), "Gelem/s"
     out = {
         "metric": "group-quant GEMM TOPS & %INT8 peak; log-quant cross-attn GB/s & %HBM",
         "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
@@ -431,11 +487,19 @@ def run_cuda(args):
         "e2e": {"value": e2e_value, "unit": "TOPS", "h2d_bytes_per_step": wl.h2d_bytes(),
                 "d2h_bytes_per_step": wl.d2h_bytes(), "ms_per_step": ms_e2e / args.steps},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "tensor", "achieved": gemm_tops, "peak": int8_peak, "unit": "TOP/s",
-                     "frac": gemm_tops / int8_peak, "traffic": gemm_traffic(),
+        "roofline": {"bound": bound, "achieved": ach, "peak": peak, "unit": unit,
+                     "frac": ach / peak, "traffic": gemm_traffic(),
+                     "frac_int8_peak": gemm_tops / int8_peak, "frac_int8_peak_burst": gemm_tops / int8_burst,
+                     "frac_own_rooflines": own_us / (gemm_ms * 1e3),
+                     "own_rooflines": "sum over the 6 launches of the slowest of each launch's tensor, HBM and "
+                                      "epilogue-conversion time, divided by the measured time",
+                     "launches": [{k: (round(v, 3) if isinstance(v, float) else v) for k, v in l.items() if k != "t_us"}
+                                  for l in launches_rf],
+                     "alu_peak": f"{CVT_PER_CLK_SM} int32->fp32 conversions per clock and SM x "
+                                 f"{props.multi_processor_count} SMs x {sm_mhz:.0f} MHz",
                      "traffic_unit": "DRAM bytes per step over the 6 launches (ncu); outputs are still in L2 when a launch ends",
                      "kernel": "gq_gemm_kernel (6 launches per step, timed on one CUDA graph of the GEMM launches of 6 consecutive steps)",
-                     "peak_source": f"2 x bf16 sustained, {peaks['source']}"},
+                     "peak_source": f"int8 = 2 x bf16 sustained, HBM = copy bandwidth, {peaks['source']}"},
         "kernels": {
             "gemm": {"ms_per_step": gemm_ms, "tops": gemm_tops, "frac_int8_peak": gemm_tops / int8_peak},
             "attention": {"ms_per_step": attn_ms, "gbs": attn_bytes() / (attn_ms * 1e-3) / 1e9,
@@ -445,6 +509,9 @@ def run_cuda(args):
         },
     }
     if rank == 0:
+        if world == 1 and not args.no_shapes:
+            # every layer shape of the five benchmark configurations, one kernel at a time
+            out["shapes"] = [time_case(torch, b, peaks, name, 5) for name in SHAPE_CASES]
         if world == 1 and not args.no_cpu_baseline:
             out["cpu_baseline"] = cpu_baseline()
         print(json.dumps(out))
@@ -510,9 +577,11 @@ def run_reference(args):
     for _ in range(max(0, min(args.warmup, 1))):
         oracle_step_sample(rows=32, attn_rows=64)
     ts, desc = [], ""
+    wall0 = time.perf_counter()
     for _ in range(max(1, min(args.steps, 3))):
         t, desc = oracle_step_sample()
         ts.append(t)
+    wall = time.perf_counter() - wall0
     t = float(np.mean(ts))
     v = gemm_ops() / t / 1e12
     print(json.dumps({
@@ -520,6 +589,8 @@ def run_reference(args):
         "value": v, "unit": "TOPS", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": len(ts),
         "warmup": max(0, min(args.warmup, 1)), "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int64/f64", "data": "synthetic", "config": {"workload": WORKLOAD},
+        # each step ran a bounded sample of the workload; ms_per_step is that time scaled to a whole step
+        "extrapolated": True, "measured_wall_seconds": wall, "steps_requested": args.steps,
         "cpu_baseline": {"value": v, "unit": "TOPS", "cores": 1, "kind": "oracle", "sample": desc},
         "e2e": {"value": v, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -552,131 +623,182 @@ MICRO_CASES = {
     "attn_8x256x160": ("attn", dict(B=8, H=8, nq=256, nk=77, d=160)),
     "attn_sdxl_1x10x1024x64": ("attn", dict(B=1, H=10, nq=1024, nk=77, d=64)),
     "gemm_sdxl_1024x5120x640_w8": ("gemm", dict(M=1024, P=1024, N=5120, C=640, G=8, wbits=8)),
+    # the remaining layer shapes of the benchmark configurations
+    "cfg1_gemm_256x320x320_w8": ("gemm", dict(M=256, P=256, N=320, C=320, G=4, wbits=8, explicit=1)),
+    "gemm_32768x320x320_w4": ("gemm", dict(M=32768, P=4096, N=320, C=320, G=8, wbits=4)),
+    "gemm_32768x2560x320_w4": ("gemm", dict(M=32768, P=4096, N=2560, C=320, G=8, wbits=4)),
+    "gemm_616x320x768_w4": ("gemm", dict(M=616, P=77, N=320, C=768, G=8, wbits=4)),
+    "gemm_616x640x768_w4": ("gemm", dict(M=616, P=77, N=640, C=768, G=8, wbits=4)),
+    "gemm_616x1280x768_w4": ("gemm", dict(M=616, P=77, N=1280, C=768, G=8, wbits=4)),
+    "gemm_2048x1280x1280_w4": ("gemm", dict(M=2048, P=256, N=1280, C=1280, G=8, wbits=4)),
+    "gemm_2048x10240x1280_w4": ("gemm", dict(M=2048, P=256, N=10240, C=1280, G=8, wbits=4)),
+    "gemm_512x1280x1280_w4": ("gemm", dict(M=512, P=64, N=1280, C=1280, G=8, wbits=4)),
+    "gemm_512x10240x1280_w4": ("gemm", dict(M=512, P=64, N=10240, C=1280, G=8, wbits=4)),
+    "gemm_512x1280x5120_w4": ("gemm", dict(M=512, P=64, N=1280, C=5120, G=8, wbits=4)),
+    "conv_8x8x8x1280": ("conv", dict(n=8, h=8, w=8, C=1280, N=1280, G=16)),
+    "attn_8x64x160": ("attn", dict(B=8, H=8, nq=64, nk=77, d=160)),
     "selfattn_2x4096x40": ("selfattn", dict(B=2, H=8, n=4096, d=40)),
     "selfattn_8x1024x80": ("selfattn", dict(B=8, H=8, n=1024, d=80)),
     "selfattn_8x256x160": ("selfattn", dict(B=8, H=8, n=256, d=160)),
 }
 
 
+# The layer shapes of the five benchmark configurations, timed one kernel at a time by the default run
+# ("shapes" in its JSON line): config 1; config 2 (W8A8, 8192 tokens); config 3 and 5 (cross-attention at the
+# four resolutions, batch 2 and 8); config 4 (W4A8 transformer linears of the four levels at batch 8); config 5
+# (W4A6 3x3 convs at batch 8).
+SHAPE_CASES = [
+    "cfg1_gemm_256x320x320_w8",
+    "gemm_8192x320x320_w8", "gemm_8192x2560x320_w8", "gemm_8192x320x1280_w8",
+    "attn_2x4096x40",
+    "gemm_32768x320x320_w4", "gemm_32768x2560x320_w4", "gemm_32768x320x1280_w4", "gemm_616x320x768_w4",
+    "gemm_8192x640x640_w4", "gemm_8192x5120x640_w4", "gemm_8192x640x2560_w4", "gemm_616x640x768_w4",
+    "gemm_2048x1280x1280_w4", "gemm_2048x10240x1280_w4", "gemm_2048x1280x5120_w4", "gemm_616x1280x768_w4",
+    "gemm_512x1280x1280_w4", "gemm_512x10240x1280_w4", "gemm_512x1280x5120_w4",
+    "conv_8x64x64x320", "conv_8x32x32x640", "conv_8x16x16x1280", "conv_8x8x8x1280",
+    "attn_8x4096x40", "attn_8x1024x80", "attn_8x256x160", "attn_8x64x160",
+    "quant_8192x320", "quant_32768x1280",
+]
+
+
+def time_case(torch, b, peaks, name, steps):
+    """Times one single-kernel case: a CUDA graph of back-to-back launches that rotate over buffer sets
+    larger than L2, replayed and timed with CUDA events (median of `steps` replays after 3 warm-up replays).
+    Returns the record with the case's own roofline: the slowest of its algorithmic bytes at the measured copy
+    bandwidth, its operations at the measured burst tensor peak and, for the GEMMs, its per-group epilogue
+    conversions at the SMs' conversion rate."""
+    kind, p = MICRO_CASES[name]
+    fns, algo_bytes, algo_ops, algo_elems = [], 0.0, 0.0, 0.0
+    if kind in ("quant", "gemm", "conv"):
+        conv = None
+        if kind == "conv":
+            P, M, C, bits, tok = p["h"] * p["w"], p["n"] * p["h"] * p["w"], p["C"], 6, False
+            conv = (p["n"], p["h"], p["w"], C)
+        else:
+            P, M, C, bits, tok = p["P"], p["M"], p["C"], 8, True
+        Xcal = torch.from_numpy(synth.activations(SEED, 100, 2, P, C, token_outliers=tok)).cuda()
+        g = b.calibrate_groups(Xcal, P, bits, p["G"], b.DIM_CHANNEL,
+                               b.OUTLIER_EXPLICIT if p.get("explicit") else b.OUTLIER_KMEANS)
+        Xh = synth.activations(SEED, 1, -(-M // P), P, C, token_outliers=tok)[:M]
+        per_set = M * C * 2 + M * g.K_pad + (M * p.get("N", 0) * 2)
+        n_sets = max(2, int(3 * 126e6 // per_set) + 1)
+        dyn = kind == "gemm" or (kind == "quant" and p["dynamic"])
+        mode = b.MODE_DYNAMIC_TOKEN if dyn else b.MODE_STATIC
+        layout = b.CODES_S8_CENTRED if kind == "conv" else b.CODES_U8
+        sets = []
+        for _ in range(n_sets):
+            X = torch.from_numpy(Xh).cuda()
+            Xq = torch.empty((M, g.K_pad), dtype=torch.uint8, device="cuda")
+            ds = torch.empty((M, g.G), dtype=torch.float32, device="cuda") if dyn else None
+            dz = torch.empty((M, g.G), dtype=torch.int32, device="cuda") if dyn else None
+            b.quantize_act_into(g, X, Xq, ds, dz, mode=mode, layout=layout)
+            Y = torch.empty((M, p["N"]), dtype=torch.float16, device="cuda") if kind != "quant" else None
+            sets.append((X, Xq, ds, dz, Y))
+        if kind == "quant":
+            fns = [lambda s=s: b.quantize_act_into(g, s[0], s[1], s[2], s[3], mode=mode, layout=layout) for s in sets]
+            algo_bytes = 3.0 * M * C + (8.0 * M * g.G if dyn else 0)
+        else:
+            if kind == "conv":
+                W = torch.from_numpy(synth.conv_weights(SEED, 2, p["N"], C)).cuda()
+                w = b.weight_prepare(g, W, 4, conv=conv)
+                kreal, wb = 9 * C, 4
+            else:
+                W = torch.from_numpy(synth.weights(SEED, 2, p["N"], C)).cuda()
+                w = b.weight_prepare(g, W, p["wbits"])
+                kreal, wb = C, p["wbits"]
+            bias = torch.from_numpy(synth.bias(SEED, 3, p["N"])).cuda()
+            ws_need = b.linear_workspace_bytes(g, w, M)      # 4-bit weights are expanded into it by every call
+            ws = torch.empty(ws_need, dtype=torch.uint8, device="cuda") if ws_need else None
+            fns = [lambda s=s: b.linear(g, w, s[1], mode=mode, layout=layout, dyn_scale=s[2], dyn_zp=s[3],
+                                        bias=bias, out=s[4], conv=conv, workspace=ws) for s in sets]
+            algo_ops = 2.0 * M * p["N"] * kreal
+            algo_bytes = M * C + p["N"] * kreal * wb / 8 + 2.0 * M * p["N"]
+            algo_elems = float(M) * p["N"] * g.G
+        extra = {"K_pad": g.K_pad, "G": g.G}
+    elif kind == "selfattn":
+        rng = np.random.default_rng(SEED)
+        shape = (p["B"], p["n"], p["H"], p["d"])
+        n_sets = max(2, int(3 * 126e6 // (4 * 2 * np.prod(shape))) + 1)
+        sets = [tuple(torch.from_numpy(rng.normal(0, 1, shape).astype(np.float16)).cuda() for _ in range(3))
+                + (torch.empty(shape, dtype=torch.float16, device="cuda"),) for _ in range(n_sets)]
+        fns = [lambda s=s: b.self_attn_logq(s[0], s[1], s[2], 8, out=s[3]) for s in sets]
+        algo_bytes = 4.0 * 2 * np.prod(shape)
+        algo_ops = 4.0 * p["B"] * p["H"] * p["n"] * p["n"] * p["d"]      # Q K^T and P V, once each
+        extra = {}
+    else:
+        a = p
+        Q, K, V = synth.attention_inputs(SEED, a["B"], a["H"], a["nq"], a["nk"], a["d"])
+        per_set = 2 * Q.size * 2
+        n_sets = max(2, int(3 * 126e6 // per_set) + 1)
+        ws_bytes = b.cross_attn_workspace_bytes(a["B"], a["H"], a["nq"], a["nk"], a["d"])
+        sets = [(torch.from_numpy(Q).cuda(), torch.from_numpy(K).cuda(), torch.from_numpy(V).cuda(),
+                 torch.empty(Q.shape, dtype=torch.float16, device="cuda"),
+                 torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")) for _ in range(n_sets)]
+        fns = [lambda s=s: b.cross_attn_logq(s[0], s[1], s[2], 8, out=s[3], workspace=s[4],
+                                             v_bits=p.get("v_bits", 0)) for s in sets]
+        algo_bytes = 2.0 * Q.size * 2 + 2.0 * K.size * 2
+        extra = {}
+    reps = max(1, 24 // len(fns))
+    for f in fns:
+        f()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            for _ in range(reps):
+                for f in fns:
+                    f()
+    n_launch = reps * len(fns)
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(3 + steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1) * 1e3 / n_launch)
+    us = float(np.median(times[3:]))
+    rec = {"case": name, "us": us, "gbs": algo_bytes / us / 1e3, "frac_hbm": algo_bytes / us / 1e3 / peaks["hbm"],
+           "sets": len(fns), **extra}
+    t_hbm_us, t_tc_us = algo_bytes / peaks["hbm"] / 1e3, 0.0
+    t_alu_us = algo_elems / alu_peak_gelems(torch.cuda.get_device_properties(0).multi_processor_count) / 1e3
+    if algo_ops:
+        rec["tops"] = algo_ops / us / 1e6
+        if kind == "selfattn":      # fp16 operands: the measured bf16 peak is the denominator
+            rec["frac_f16_peak"] = rec["tops"] / peaks["bf16"]
+            t_tc_us = algo_ops / peaks["bf16"] / 1e6
+        else:
+            rec["frac_int8_peak"] = rec["tops"] / (2 * peaks["bf16"])
+            t_tc_us = algo_ops / (2 * peaks["bf16"]) / 1e6
+    t = {"tensor": t_tc_us, "hbm": t_hbm_us, "alu": t_alu_us}
+    rec["bound"] = max(t, key=t.get)
+    rec["roofline_us"] = t[rec["bound"]]
+    rec["frac_roofline"] = rec["roofline_us"] / us
+    assert b.device_status() == 0
+    del sets, fns, graph
+    return {k: (round(v, 4) if isinstance(v, float) else v) for k, v in rec.items()}
+
+
 def run_micro(args):
-    """Times single kernels: each case is captured as a CUDA graph of back-to-back launches that
-    rotate over buffer sets larger than L2, replayed and timed with CUDA events."""
+    """Times single kernels (see time_case) and prints one JSON line per case."""
     import torch
     from paper_2501_04304_b200 import binding as b
     torch.cuda.set_device(0)
     peaks = measured_peaks()
-    names = [n for n in MICRO_CASES if args.micro == "all" or n.startswith(args.micro)]
-    for name in names:
-        kind, p = MICRO_CASES[name]
-        fns, algo_bytes, algo_ops = [], 0.0, 0.0
-        if kind in ("quant", "gemm", "conv"):
-            conv = None
-            if kind == "conv":
-                P, M, C, bits, tok = p["h"] * p["w"], p["n"] * p["h"] * p["w"], p["C"], 6, False
-                conv = (p["n"], p["h"], p["w"], C)
-            else:
-                P, M, C, bits, tok = p["P"], p["M"], p["C"], 8, True
-            Xcal = torch.from_numpy(synth.activations(SEED, 100, 2, P, C, token_outliers=tok)).cuda()
-            g = b.calibrate_groups(Xcal, P, bits, p["G"], b.DIM_CHANNEL)
-            Xh = synth.activations(SEED, 1, M // P, P, C, token_outliers=tok)
-            per_set = M * C * 2 + M * g.K_pad + (M * p.get("N", 0) * 2)
-            n_sets = max(2, int(3 * 126e6 // per_set) + 1)
-            dyn = kind == "gemm" or (kind == "quant" and p["dynamic"])
-            mode = b.MODE_DYNAMIC_TOKEN if dyn else b.MODE_STATIC
-            layout = b.CODES_S8_CENTRED if kind == "conv" else b.CODES_U8
-            sets = []
-            for _ in range(n_sets):
-                X = torch.from_numpy(Xh).cuda()
-                Xq = torch.empty((M, g.K_pad), dtype=torch.uint8, device="cuda")
-                ds = torch.empty((M, g.G), dtype=torch.float32, device="cuda") if dyn else None
-                dz = torch.empty((M, g.G), dtype=torch.int32, device="cuda") if dyn else None
-                b.quantize_act_into(g, X, Xq, ds, dz, mode=mode, layout=layout)
-                Y = torch.empty((M, p["N"]), dtype=torch.float16, device="cuda") if kind != "quant" else None
-                sets.append((X, Xq, ds, dz, Y))
-            if kind == "quant":
-                fns = [lambda s=s: b.quantize_act_into(g, s[0], s[1], s[2], s[3], mode=mode, layout=layout) for s in sets]
-                algo_bytes = 3.0 * M * C + (8.0 * M * g.G if dyn else 0)
-            else:
-                if kind == "conv":
-                    W = torch.from_numpy(synth.conv_weights(SEED, 2, p["N"], C)).cuda()
-                    w = b.weight_prepare(g, W, 4, conv=conv)
-                    kreal, wb = 9 * C, 4
-                else:
-                    W = torch.from_numpy(synth.weights(SEED, 2, p["N"], C)).cuda()
-                    w = b.weight_prepare(g, W, p["wbits"])
-                    kreal, wb = C, p["wbits"]
-                bias = torch.from_numpy(synth.bias(SEED, 3, p["N"])).cuda()
-                ws_need = b.linear_workspace_bytes(g, w, M)      # 4-bit weights are expanded into it by every call
-                ws = torch.empty(ws_need, dtype=torch.uint8, device="cuda") if ws_need else None
-                fns = [lambda s=s: b.linear(g, w, s[1], mode=mode, layout=layout, dyn_scale=s[2], dyn_zp=s[3],
-                                            bias=bias, out=s[4], conv=conv, workspace=ws) for s in sets]
-                algo_ops = 2.0 * M * p["N"] * kreal
-                algo_bytes = M * C + p["N"] * kreal * wb / 8 + 2.0 * M * p["N"]
-            extra = {"K_pad": g.K_pad, "G": g.G}
-        elif kind == "selfattn":
-            rng = np.random.default_rng(SEED)
-            shape = (p["B"], p["n"], p["H"], p["d"])
-            n_sets = max(2, int(3 * 126e6 // (4 * 2 * np.prod(shape))) + 1)
-            sets = [tuple(torch.from_numpy(rng.normal(0, 1, shape).astype(np.float16)).cuda() for _ in range(3))
-                    + (torch.empty(shape, dtype=torch.float16, device="cuda"),) for _ in range(n_sets)]
-            fns = [lambda s=s: b.self_attn_logq(s[0], s[1], s[2], 8, out=s[3]) for s in sets]
-            algo_bytes = 4.0 * 2 * np.prod(shape)
-            algo_ops = 4.0 * p["B"] * p["H"] * p["n"] * p["n"] * p["d"]      # Q K^T and P V, once each
-            extra = {}
-        else:
-            a = p
-            Q, K, V = synth.attention_inputs(SEED, a["B"], a["H"], a["nq"], a["nk"], a["d"])
-            per_set = 2 * Q.size * 2
-            n_sets = max(2, int(3 * 126e6 // per_set) + 1)
-            ws_bytes = b.cross_attn_workspace_bytes(a["B"], a["H"], a["nq"], a["nk"], a["d"])
-            sets = [(torch.from_numpy(Q).cuda(), torch.from_numpy(K).cuda(), torch.from_numpy(V).cuda(),
-                     torch.empty(Q.shape, dtype=torch.float16, device="cuda"),
-                     torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")) for _ in range(n_sets)]
-            fns = [lambda s=s: b.cross_attn_logq(s[0], s[1], s[2], 8, out=s[3], workspace=s[4],
-                                                 v_bits=p.get("v_bits", 0)) for s in sets]
-            algo_bytes = 2.0 * Q.size * 2 + 2.0 * K.size * 2
-            extra = {}
-        reps = max(1, 24 // len(fns))
-        for f in fns:
-            f()
-        torch.cuda.synchronize()
-        graph = torch.cuda.CUDAGraph()
-        stream = torch.cuda.Stream()
-        with torch.cuda.stream(stream):
-            with torch.cuda.graph(graph, stream=stream):
-                for _ in range(reps):
-                    for f in fns:
-                        f()
-        n_launch = reps * len(fns)
-        torch.cuda.synchronize()
-        times = []
-        for _ in range(3 + args.steps):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            graph.replay()
-            e1.record()
-            torch.cuda.synchronize()
-            times.append(e0.elapsed_time(e1) * 1e3 / n_launch)
-        us = float(np.median(times[3:]))
-        rec = {"case": name, "us": us, "gbs": algo_bytes / us / 1e3, "frac_hbm": algo_bytes / us / 1e3 / peaks["hbm"],
-               "sets": len(fns), **extra}
-        t_hbm_us, t_tc_us = algo_bytes / peaks["hbm"] / 1e3, 0.0
-        if algo_ops:
-            rec["tops"] = algo_ops / us / 1e6
-            if kind == "selfattn":      # fp16 operands: the measured bf16 peak is the denominator
-                rec["frac_f16_peak"] = rec["tops"] / peaks["bf16"]
-                t_tc_us = algo_ops / peaks["bf16"] / 1e6
-            else:
-                rec["frac_int8_peak"] = rec["tops"] / (2 * peaks["bf16"])
-                t_tc_us = algo_ops / (2 * peaks["bf16"]) / 1e6
-        # the shape's own roofline: the slower of its algorithmic bytes at the measured copy bandwidth and its
-        # algorithmic operations at the measured (burst) tensor peak
-        rec["bound"] = "tensor" if t_tc_us > t_hbm_us else "hbm"
-        rec["roofline_us"] = max(t_tc_us, t_hbm_us)
-        rec["frac_roofline"] = rec["roofline_us"] / us
-        assert b.device_status() == 0
-        print(json.dumps(rec), flush=True)
-        del sets, fns, graph
+    for name in [n for n in MICRO_CASES if args.micro == "all" or n.startswith(args.micro)]:
+        print(json.dumps(time_case(torch, b, peaks, name, args.steps)), flush=True)
+
+
+def rank_launch_command(n, argv):
+    """The command that runs this script as n ranks of one node (replicas only), one GPU each."""
+    import socket
+    with socket.socket() as so:
+        so.bind(("127.0.0.1", 0))
+        port = so.getsockname()[1]
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
 
 
 def main():
@@ -686,8 +808,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-shapes", action="store_true", help="skip the per-shape single-kernel timings")
     ap.add_argument("--micro", default=None, help="time single kernels: 'all' or a case-name prefix")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.micro:
+        # started without a launcher: start one rank per GPU of this node and let them print the line
+        sys.exit(subprocess.call(rank_launch_command(args.gpus, sys.argv[1:])))
     if args.micro:
         run_micro(args)
     elif args.impl == "reference":

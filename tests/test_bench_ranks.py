@@ -83,3 +83,23 @@ def test_reference_arm_runs_on_rank0_only():
     assert rec["e2e"] == {"value": rec["value"], "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
     assert rec["cpu_baseline"]["kind"] == "oracle" and rec["cpu_baseline"]["value"] == rec["value"]
     assert lines0[-1] == "CALLS 3"                            # one warm-up and two timed samples
+
+
+def test_gpus_flag_without_a_launcher_starts_the_ranks_itself():
+    """`bench.py --gpus 2` started plainly (no WORLD_SIZE) re-runs itself as two ranks of one node; shown here with
+    the oracle arm, which needs no GPU: one JSON line, from rank 0, that says n_gpus = 2."""
+    sys.path.insert(0, ROOT)
+    import bench
+    cmd = bench.rank_launch_command(2, ["--gpus", "2"])
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"] and "--nproc-per-node=2" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[-2:] == ["--gpus", "2"]
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference",
+                          "--steps", "1", "--warmup", "0"], env=env, cwd=ROOT, capture_output=True, text=True,
+                         timeout=600)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    rec = json.loads(lines[0])
+    assert rec["impl"] == "reference" and rec["n_gpus"] == 2 and rec["extrapolated"] is True
+    assert rec["measured_wall_seconds"] > 0
