@@ -19,6 +19,8 @@
 // served by L2), K and V once per CTA from L2.
 #pragma once
 
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 
 namespace dgq {
@@ -135,6 +137,17 @@ __device__ __forceinline__ void stage_q(const __half* q_base, int64_t q_stride, 
   __syncwarp();
 }
 
+// Four 8 x 8 fp16 matrices from shared memory: lane l gives the address of row l % 8 of matrix l / 8 (16 bytes,
+// 16-byte aligned); register i of every lane holds its two elements of matrix i in the MMA fragment layout.
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&x)[4], const __half* row) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(x[0]), "=r"(x[1]), "=r"(x[2]), "=r"(x[3])
+               : "r"(smem_u32(row)));
+}
+__device__ __forceinline__ void ldmatrix_x2(uint32_t (&x)[2], const __half* row) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0, %1}, [%2];" : "=r"(x[0]), "=r"(x[1]) : "r"(smem_u32(row)));
+}
+
 // Base-2 logits of the warp's rows against all keys.  S[mt][nt][0..1]: row 16 mt + lane/4, keys
 // 8 nt + 2 (lane%4) + {0,1}; S[mt][nt][2..3]: row + 8.  Keys >= nk get -inf.
 template <int D, int NKP>
@@ -149,22 +162,25 @@ __device__ __forceinline__ void logits_warp(const AttnArgs& a, const __half* sla
     for (int nt = 0; nt < Cfg::NT; ++nt)
 #pragma unroll
       for (int i = 0; i < 4; ++i) S[mt][nt][i] = 0.f;
+  // fragment addresses of this lane: matrix lane / 8, row lane % 8.  A: matrices (rows 0-7 | 8-15) x (k 0-7 | 8-15);
+  // B: matrices (keys of tile nt | nt + 1) x (k 0-7 | 8-15) -- the key rows of K are the columns of the operand.
+  const int lm = lane >> 3, lr = lane & 7;
+  const __half* a_row = slab + ((lm & 1) * 8 + lr) * Cfg::LDK + (lm >> 1) * 8;
+  const __half* b_row = sK + ((lm >> 1) * 8 + lr) * Cfg::LDK + (lm & 1) * 8;
 #pragma unroll
   for (int kk = 0; kk < Cfg::KS; ++kk) {
     uint32_t af[Cfg::MT][4];
 #pragma unroll
-    for (int mt = 0; mt < Cfg::MT; ++mt)
+    for (int mt = 0; mt < Cfg::MT; ++mt) ldmatrix_x4(af[mt], a_row + mt * 16 * Cfg::LDK + kk * 16);
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
-        af[mt][i] = *reinterpret_cast<const uint32_t*>(slab + (mt * 16 + r + (i & 1) * 8) * Cfg::LDK + kk * 16 +
-                                                       2 * c + (i >> 1) * 8);
+    for (int nt = 0; nt < Cfg::NT; nt += 2) {
+      uint32_t bf[4];
+      ldmatrix_x4(bf, b_row + nt * 8 * Cfg::LDK + kk * 16);
 #pragma unroll
-    for (int nt = 0; nt < Cfg::NT; ++nt) {
-      const __half* kp = sK + (nt * 8 + r) * Cfg::LDK + kk * 16 + 2 * c;
-      const uint32_t b0 = *reinterpret_cast<const uint32_t*>(kp);
-      const uint32_t b1 = *reinterpret_cast<const uint32_t*>(kp + 8);
-#pragma unroll
-      for (int mt = 0; mt < Cfg::MT; ++mt) mma_f16(S[mt][nt], af[mt][0], af[mt][1], af[mt][2], af[mt][3], b0, b1);
+      for (int mt = 0; mt < Cfg::MT; ++mt) {
+        mma_f16(S[mt][nt], af[mt][0], af[mt][1], af[mt][2], af[mt][3], bf[0], bf[1]);
+        mma_f16(S[mt][nt + 1], af[mt][0], af[mt][1], af[mt][2], af[mt][3], bf[2], bf[3]);
+      }
     }
   }
 #pragma unroll
@@ -445,17 +461,30 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_phase2_kernel(const AttnAr
     for (int nt = 0; nt < NT_O; ++nt)
 #pragma unroll
       for (int i = 0; i < 4; ++i) acc[mt][nt][i] = 0.f;
+  {
+    const int lm = lane >> 3, lr = lane & 7;  // matrix and row this lane addresses
+    const __half* v_row = sVt + ((lm >> 1) * 8 + lr) * Cfg::LDV + (lm & 1) * 8;
 #pragma unroll
-  for (int kk = 0; kk < NKP; ++kk)
+    for (int kk = 0; kk < NKP; ++kk) {
 #pragma unroll
-    for (int nt = 0; nt < NT_O; ++nt) {
-      const __half* vp = sVt + (nt * 8 + r) * Cfg::LDV + kk * 16 + 2 * c;
-      const uint32_t b0 = *reinterpret_cast<const uint32_t*>(vp);
-      const uint32_t b1 = *reinterpret_cast<const uint32_t*>(vp + 8);
+      for (int nt = 0; nt + 1 < NT_O; nt += 2) {
+        uint32_t bf[4];
+        ldmatrix_x4(bf, v_row + nt * 8 * Cfg::LDV + kk * 16);
 #pragma unroll
-      for (int mt = 0; mt < Cfg::MT; ++mt)
-        mma_f16(acc[mt][nt], pa[mt][kk][0], pa[mt][kk][1], pa[mt][kk][2], pa[mt][kk][3], b0, b1);
+        for (int mt = 0; mt < Cfg::MT; ++mt) {
+          mma_f16(acc[mt][nt], pa[mt][kk][0], pa[mt][kk][1], pa[mt][kk][2], pa[mt][kk][3], bf[0], bf[1]);
+          mma_f16(acc[mt][nt + 1], pa[mt][kk][0], pa[mt][kk][1], pa[mt][kk][2], pa[mt][kk][3], bf[2], bf[3]);
+        }
+      }
+      if (NT_O & 1) {  // the last 8 features alone (lanes 16-31 repeat the addresses of lanes 0-15, unused)
+        uint32_t bf[2];
+        ldmatrix_x2(bf, v_row - (lm >> 1) * 8 * Cfg::LDV + (NT_O - 1) * 8 * Cfg::LDV + kk * 16);
+#pragma unroll
+        for (int mt = 0; mt < Cfg::MT; ++mt)
+          mma_f16(acc[mt][NT_O - 1], pa[mt][kk][0], pa[mt][kk][1], pa[mt][kk][2], pa[mt][kk][3], bf[0], bf[1]);
+      }
     }
+  }
   // O = A_i0 V_0 + s 2^-14 acc, staged in the warp's slab and written with 128-bit stores
   const float s_out = exp2f(log2s - AT_P_SHIFT);
 #pragma unroll
@@ -480,23 +509,362 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_phase2_kernel(const AttnAr
   }
 }
 
+// The two passes as one kernel: the logits and the row statistics stay in registers while the CTAs exchange
+// their maxima through the workspace and meet at the grid barrier, so Q K^T, the K / Q staging and the
+// statistics round trip happen once.  Launched cooperatively (every CTA resident) when the scale is dynamic;
+// with a fixed scale no CTA waits for another and the launch is an ordinary one.
+template <int D, int NKP, bool CODES>
+__global__ void __launch_bounds__(AT_THREADS, 2) attn_fused_kernel(const AttnArgs a) {
+  using Cfg = AttnCfg<D, NKP>;
+  constexpr int NT_O = D / 8;
+  extern __shared__ __align__(16) unsigned char at_smem[];
+  __half* sK = reinterpret_cast<__half*>(at_smem);
+  __half* sQ = reinterpret_cast<__half*>(at_smem + Cfg::SM_K);
+  __half* sVt = reinterpret_cast<__half*>(at_smem + Cfg::SM_K + Cfg::SM_Q);  // [D][LDV], column 0 zero
+  float* sV0 = reinterpret_cast<float*>(sVt + D * Cfg::LDV);                 // [D] the <start> value row
+  const int blk = blockIdx.x;
+  const int rb = blk % a.n_row_blocks;
+  const int h = (blk / a.n_row_blocks) % a.H;
+  const int b = blk / (a.n_row_blocks * a.H);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = lane >> 2, c = lane & 3;
+  const int row0 = rb * Cfg::ROWS + warp * Cfg::WROWS;
+  const int rows_valid = min(Cfg::WROWS, a.nq - row0);
+  const int64_t q_stride = (int64_t)a.H * D;
+  __half* slab = sQ + warp * Cfg::WROWS * Cfg::LDK;
+  pdl_launch_dependents();
+  pdl_wait();  // Q, K, V may come from earlier kernels
+  uint4 xk[KStage<D, NKP>::N];
+  load_k<D, NKP>(a, b, h, xk);
+  // V^T: 128-bit loads of 8 features of one key, written transposed; keys >= nk and key 0 are zero.
+  // Consecutive lanes take consecutive keys of the same 8 features, so that the transposed 2-byte stores
+  // of a warp fall into consecutive words of one V^T row (the head's V slab is a few KB and sits in L2,
+  // so the strided reads cost little).  K, V and Q are all requested before anything is written, so
+  // their latencies overlap.
+  // V is first needed after the scope's CTAs have met.  A slab of a few registers is requested up front with K
+  // and Q; a larger one is requested once the logits are there (the registers of the Q K^T fragments are free
+  // again) and arrives while the row statistics and the meeting take their time.
+  constexpr int NV = (NKP * 16 * (D / 8) + AT_THREADS - 1) / AT_THREADS;
+  constexpr bool V_EARLY = NV <= 2;
+  uint4 xv[NV];
+  auto request_v = [&]() {
+#pragma unroll
+    for (int e = 0; e < NV; ++e) {
+      const int i = threadIdx.x + e * AT_THREADS;
+      const int v = i / (NKP * 16), j = i - v * (NKP * 16);
+      xv[e] = make_uint4(0, 0, 0, 0);
+      if (j < a.nk && v < D / 8)
+        xv[e] = __ldg(reinterpret_cast<const uint4*>(a.V + (((int64_t)b * a.nk + j) * a.H + h) * D) + v);
+    }
+  };
+  if (V_EARLY) request_v();
+  // The scope's scale: its CTAs' partial maxima lie next to each other (row blocks of a head, heads of a
+  // prompt, prompts of the call); each thread takes a strided share, the warps meet after the barrier below.
+  __shared__ float part_w[AT_WARPS];
+  if (rows_valid > 0) stage_q<D, NKP>(a.Q + (((int64_t)b * a.nq + row0) * a.H + h) * D, q_stride, rows_valid, slab);
+  store_k<D, NKP>(xk, sK);
+  __syncthreads();
+  const int scope = scope_index(a, b, h);
+  // Logits once; they stay in registers across the meeting of the scope's CTAs.
+  float S[Cfg::MT][Cfg::NT][4];
+  float st_max[Cfg::MT][2], st_lz[Cfg::MT][2];  // row maximum and log2 of the row sum, rows r and r + 8 of every tile
+  float best = -INFINITY;
+  if (rows_valid > 0) logits_warp<D, NKP>(a, slab, sK, S);
+  if (!V_EARLY) request_v();
+  if (rows_valid > 0) {
+#pragma unroll
+    for (int mt = 0; mt < Cfg::MT; ++mt)
+#pragma unroll
+      for (int hi = 0; hi < 2; ++hi) {
+        float tmax = -INFINITY, trest = -INFINITY;
+#pragma unroll
+        for (int nt = 0; nt < Cfg::NT; ++nt)
+#pragma unroll
+          for (int i = 0; i < 2; ++i) {
+            const float t = S[mt][nt][hi * 2 + i];
+            if (nt == 0 && i == 0) {
+              tmax = fmaxf(tmax, t);
+              if (c != 0) trest = fmaxf(trest, t);  // key 0 (lane c == 0) is the <start> column
+            } else {
+              trest = fmaxf(trest, t);
+            }
+          }
+        tmax = fmaxf(tmax, trest);
+        tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+        tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+        trest = fmaxf(trest, __shfl_xor_sync(0xffffffffu, trest, 1));
+        trest = fmaxf(trest, __shfl_xor_sync(0xffffffffu, trest, 2));
+        float z = 0.f;
+#pragma unroll
+        for (int nt = 0; nt < Cfg::NT; ++nt)
+#pragma unroll
+          for (int i = 0; i < 2; ++i) z += ex2_approx(S[mt][nt][hi * 2 + i] - tmax);
+        z += __shfl_xor_sync(0xffffffffu, z, 1);
+        z += __shfl_xor_sync(0xffffffffu, z, 2);
+        const float lz = log2f(z);
+        st_max[mt][hi] = tmax;
+        st_lz[mt][hi] = lz;
+        if (mt * 16 + r + hi * 8 < rows_valid) best = fmaxf(best, (trest - tmax) - lz);  // log2 of the row's largest off-<start> score
+      }
+  }
+  __syncwarp();  // the slab is reused for the output rows below
+  // The scope's scale: every CTA leaves its maximum in its own word, all CTAs of the grid meet (the grid is
+  // launched cooperatively, so all of them are resident and the runtime's grid barrier applies), then every CTA
+  // reduces the words of its scope.  The V^T operand is staged between the store and the meeting.
+  if (!a.fixed_scale) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, o));
+    if (lane == 0) part_w[warp] = best;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+#pragma unroll
+      for (int w = 1; w < AT_WARPS; ++w) best = fmaxf(best, part_w[w]);
+      a.part[((int64_t)b * a.H + h) * a.n_row_blocks + rb] = best;
+    }
+  }
+  // Quantized value operand: range of the head's slab (every CTA of the head derives the same
+  // parameters), codes decided in fp32, de-quantized as s (q - Z); rows j >= 1 become the fp16
+  // operand of the product, row 0 stays fp32.
+  float v_s = 0.f, v_inv = 0.f, v_Zf = 0.f, v_L = 0.f;
+  if (a.v_bits) {
+    __shared__ float v_red[2 * (AT_THREADS / 32)];
+    float lo = INFINITY, hi = -INFINITY;
+#pragma unroll
+    for (int ev = 0; ev < NV; ++ev) {
+      const int i = threadIdx.x + ev * AT_THREADS;
+      if (i % (NKP * 16) < a.nk && i < NKP * 16 * (D / 8)) {
+        const __half* xh = reinterpret_cast<const __half*>(&xv[ev]);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float f = __half2float(xh[e]);
+          lo = fminf(lo, f);
+          hi = fmaxf(hi, f);
+        }
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+      hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    if (lane == 0) {
+      v_red[warp] = lo;
+      v_red[AT_THREADS / 32 + warp] = hi;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < AT_THREADS / 32; ++w) {
+      lo = fminf(lo, v_red[w]);
+      hi = fmaxf(hi, v_red[AT_THREADS / 32 + w]);
+    }
+    int v_Z;
+    group_params(lo, hi, a.v_bits, v_s, v_inv, v_Z);
+    v_Zf = (float)v_Z;
+    v_L = (float)((1 << a.v_bits) - 1);
+  }
+#pragma unroll
+  for (int ev = 0; ev < NV; ++ev) {
+    const int i = threadIdx.x + ev * AT_THREADS;
+    if (i >= NKP * 16 * (D / 8)) continue;
+    const int v = i / (NKP * 16), j = i - v * (NKP * 16);
+    const __half* xh = reinterpret_cast<const __half*>(&xv[ev]);
+    float f[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      f[e] = __half2float(xh[e]);
+      if (a.v_bits && j < a.nk)
+        f[e] = __fmul_rn(v_s, __fsub_rn((float)quantize_code(f[e], v_inv, v_Zf, v_L), v_Zf));
+    }
+    if (j == 0) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        sV0[v * 8 + e] = f[e];
+        sVt[(v * 8 + e) * Cfg::LDV] = __float2half(0.f);
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) sVt[(v * 8 + e) * Cfg::LDV + j] = __float2half_rn(f[e]);
+    }
+  }
+  float log2s;
+  if (a.fixed_scale) {
+    log2s = log2f(fmaxf(__ldg(a.fixed_scale + scope), 1.17549435e-38f));
+    __syncthreads();  // V^T is staged
+  } else {
+    cooperative_groups::this_grid().sync();  // every CTA's maximum is written and visible; V^T is staged
+    const int per_head = a.n_row_blocks;
+    const int64_t first = a.gran == DGQ_SCALE_PER_PROMPT ? (int64_t)b * a.H * per_head
+                          : (a.gran == DGQ_SCALE_PER_PROMPT_HEAD ? ((int64_t)b * a.H + h) * per_head : 0);
+    const int count = a.gran == DGQ_SCALE_PER_PROMPT ? a.H * per_head
+                      : (a.gran == DGQ_SCALE_PER_PROMPT_HEAD ? per_head : a.B * a.H * per_head);
+    float m = -INFINITY;
+    for (int i = threadIdx.x; i < count; i += AT_THREADS) m = fmaxf(m, __ldcg(a.part + first + i));  // written by this grid: L2
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0) part_w[warp] = m;  // (free again: the grid barrier is also a barrier of the CTA)
+    __syncthreads();
+    log2s = part_w[0];
+#pragma unroll
+    for (int w = 1; w < AT_WARPS; ++w) log2s = fmaxf(log2s, part_w[w]);
+  }
+  if (a.scale_out && threadIdx.x == 0 && rb == 0 &&
+      (a.gran == DGQ_SCALE_PER_PROMPT_HEAD || (a.gran == DGQ_SCALE_PER_PROMPT && h == 0) || (b == 0 && h == 0)))
+    a.scale_out[scope] = exp2f(log2s);
+  if (rows_valid <= 0) return;
+
+  const float Lf = (float)((1 << a.bits) - 1);
+  const float Lcap = fminf(Lf, AT_CODE_CAP);
+  uint32_t pa[Cfg::MT][NKP][4];  // A fragments of A_hat / s * 2^14 for the second product
+  float a0[Cfg::MT][2];          // the <start> score of rows r and r + 8
+#pragma unroll
+  for (int mt = 0; mt < Cfg::MT; ++mt)
+#pragma unroll
+    for (int hi = 0; hi < 2; ++hi) {
+      const float2 st = make_float2(st_max[mt][hi], st_lz[mt][hi]);
+      const float base = log2s + st.x + st.y;  // code = rint(base - t)
+      float start = ex2_approx(S[mt][0][hi * 2] - st.x - st.y);  // meaningful on the lane with c == 0
+      a0[mt][hi] = __shfl_sync(0xffffffffu, start, lane & ~3);
+#pragma unroll
+      for (int nt = 0; nt < Cfg::NT; ++nt) {
+        float p[2];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const float t = S[mt][nt][hi * 2 + i];
+          // rint by adding 1.5 * 2^23: the low bits of the sum are the integer.  -inf logits (padding
+          // keys) clamp to the cap; their V^T columns are zero, as is the <start> column.
+          const float x = fminf(fmaxf(base - t, 0.f), CODES ? Lf : Lcap);
+          const uint32_t bits = __float_as_uint(x + 12582912.0f);  // 0x4B400000 + code
+          if (CODES) {
+            const int key = nt * 8 + 2 * c + i;
+            const int orow = mt * 16 + r + hi * 8;
+            if (key >= 1 && key < a.nk && orow < rows_valid)
+              a.codes_out[(((int64_t)b * a.H + h) * a.nq + row0 + orow) * (a.nk - 1) + key - 1] = (uint8_t)(bits & 0xFFu);
+          }
+          // 2^(14 - code) as an fp32 exponent field: (127 + 14 - code) << 23, where the shift drops the
+          // 0x4B400000 of `bits` (its low 9 bits are zero).  Without the code output x is already held
+          // to the cap, beyond which the product would convert to an fp16 zero anyway.
+          const uint32_t capped = CODES ? min(bits, 0x4B400000u + (uint32_t)AT_CODE_CAP) : bits;
+          p[i] = __uint_as_float(((127u + (uint32_t)AT_P_SHIFT) << 23) - (capped << 23));
+        }
+        const __half2 ph = __floats2half2_rn(p[0], p[1]);
+        pa[mt][nt >> 1][(nt & 1) * 2 + hi] = *reinterpret_cast<const uint32_t*>(&ph);
+      }
+    }
+  float acc[Cfg::MT][NT_O][4];
+#pragma unroll
+  for (int mt = 0; mt < Cfg::MT; ++mt)
+#pragma unroll
+    for (int nt = 0; nt < NT_O; ++nt)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) acc[mt][nt][i] = 0.f;
+  {
+    const int lm = lane >> 3, lr = lane & 7;  // matrix and row this lane addresses
+    const __half* v_row = sVt + ((lm >> 1) * 8 + lr) * Cfg::LDV + (lm & 1) * 8;
+#pragma unroll
+    for (int kk = 0; kk < NKP; ++kk) {
+#pragma unroll
+      for (int nt = 0; nt + 1 < NT_O; nt += 2) {
+        uint32_t bf[4];
+        ldmatrix_x4(bf, v_row + nt * 8 * Cfg::LDV + kk * 16);
+#pragma unroll
+        for (int mt = 0; mt < Cfg::MT; ++mt) {
+          mma_f16(acc[mt][nt], pa[mt][kk][0], pa[mt][kk][1], pa[mt][kk][2], pa[mt][kk][3], bf[0], bf[1]);
+          mma_f16(acc[mt][nt + 1], pa[mt][kk][0], pa[mt][kk][1], pa[mt][kk][2], pa[mt][kk][3], bf[2], bf[3]);
+        }
+      }
+      if (NT_O & 1) {  // the last 8 features alone (lanes 16-31 repeat the addresses of lanes 0-15, unused)
+        uint32_t bf[2];
+        ldmatrix_x2(bf, v_row - (lm >> 1) * 8 * Cfg::LDV + (NT_O - 1) * 8 * Cfg::LDV + kk * 16);
+#pragma unroll
+        for (int mt = 0; mt < Cfg::MT; ++mt)
+          mma_f16(acc[mt][NT_O - 1], pa[mt][kk][0], pa[mt][kk][1], pa[mt][kk][2], pa[mt][kk][3], bf[0], bf[1]);
+      }
+    }
+  }
+  // O = A_i0 V_0 + s 2^-14 acc, staged in the warp's slab and written with 128-bit stores
+  const float s_out = exp2f(log2s - AT_P_SHIFT);
+#pragma unroll
+  for (int nt = 0; nt < NT_O; ++nt) {
+    const int col = nt * 8 + 2 * c;
+    const float2 v0 = *reinterpret_cast<const float2*>(sV0 + col);
+#pragma unroll
+    for (int mt = 0; mt < Cfg::MT; ++mt)
+#pragma unroll
+      for (int hi = 0; hi < 2; ++hi) {
+        const float ox = fmaf(a0[mt][hi], v0.x, s_out * acc[mt][nt][hi * 2]);
+        const float oy = fmaf(a0[mt][hi], v0.y, s_out * acc[mt][nt][hi * 2 + 1]);
+        *reinterpret_cast<__half2*>(slab + (mt * 16 + r + hi * 8) * Cfg::LDK + col) = __floats2half2_rn(ox, oy);
+      }
+  }
+  __syncwarp();
+  __half* o_base = a.O + (((int64_t)b * a.nq + row0) * a.H + h) * D;
+  for (int i = lane; i < Cfg::WROWS * (D / 8); i += 32) {
+    const int rr = i / (D / 8), v = i - rr * (D / 8);
+    if (rr < rows_valid)
+      *(reinterpret_cast<uint4*>(o_base + rr * q_stride) + v) = *reinterpret_cast<const uint4*>(slab + rr * Cfg::LDK + v * 8);
+  }
+}
+
+// Launch with the cooperative attribute: every CTA of the grid is resident at the same time (the launch
+// fails instead of running a grid that is not), which the fused kernel's meeting of CTAs relies on.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_cooperative(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                      Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 template <int D, int NKP>
-static dgq_status launch_attn(const AttnArgs& a, cudaStream_t stream) {
+static dgq_status launch_attn(const AttnArgs& a, bool allow_fused, cudaStream_t stream) {
   using Cfg = AttnCfg<D, NKP>;
   constexpr int SM1 = Cfg::SMEM1;
   constexpr int SM2 = Cfg::SMEM2;
-  static bool attr_set[64] = {false};
+  static std::atomic<int> capacity[64];  // CTAs of the fused kernel that fit the device at once; 0 = not asked yet
   int dev = 0;
   DGQ_CUDA_OK(cudaGetDevice(&dev));
-  if (dev >= 64 || !attr_set[dev]) {
+  if (dev < 0 || dev >= 64) return DGQ_ERR_UNSUPPORTED;
+  if (capacity[dev].load() == 0) {
     DGQ_CUDA_OK(cudaFuncSetAttribute(attn_phase1_kernel<D, NKP>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM1));
     DGQ_CUDA_OK(cudaFuncSetAttribute(attn_phase2_kernel<D, NKP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM2));
     DGQ_CUDA_OK(cudaFuncSetAttribute(attn_phase2_kernel<D, NKP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM2));
-    if (dev < 64) attr_set[dev] = true;
+    DGQ_CUDA_OK(cudaFuncSetAttribute(attn_fused_kernel<D, NKP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM2));
+    DGQ_CUDA_OK(cudaFuncSetAttribute(attn_fused_kernel<D, NKP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM2));
+    int n_sm = 0, per_sm0 = 0, per_sm1 = 0;
+    DGQ_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+    DGQ_CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm0, attn_fused_kernel<D, NKP, false>, AT_THREADS, SM2));
+    DGQ_CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm1, attn_fused_kernel<D, NKP, true>, AT_THREADS, SM2));
+    capacity[dev].store(std::max(1, n_sm * std::min(per_sm0, per_sm1)));
   }
   AttnArgs aa = a;
   aa.n_row_blocks = (a.nq + Cfg::ROWS - 1) / Cfg::ROWS;
   const int grid = a.B * a.H * aa.n_row_blocks;
+  if (allow_fused && (a.fixed_scale != nullptr || grid <= capacity[dev].load())) {
+    // one kernel: with a fixed scale its CTAs never wait for one another; with a dynamic one they meet at the
+    // grid barrier, and the launch guarantees that all of them are resident
+    if (a.fixed_scale) {
+      if (a.codes_out)
+        DGQ_CUDA_OK(launch_pdl(attn_fused_kernel<D, NKP, true>, dim3(grid), dim3(AT_THREADS), (size_t)SM2, stream, aa));
+      else
+        DGQ_CUDA_OK(launch_pdl(attn_fused_kernel<D, NKP, false>, dim3(grid), dim3(AT_THREADS), (size_t)SM2, stream, aa));
+    } else {
+      if (a.codes_out)
+        DGQ_CUDA_OK(launch_cooperative(attn_fused_kernel<D, NKP, true>, dim3(grid), dim3(AT_THREADS), (size_t)SM2, stream, aa));
+      else
+        DGQ_CUDA_OK(launch_cooperative(attn_fused_kernel<D, NKP, false>, dim3(grid), dim3(AT_THREADS), (size_t)SM2, stream, aa));
+    }
+    g_launches += 1;
+    DGQ_CUDA_OK(cudaGetLastError());
+    return DGQ_OK;
+  }
   DGQ_CUDA_OK(launch_pdl(attn_phase1_kernel<D, NKP>, dim3(grid), dim3(AT_THREADS), (size_t)SM1, stream, aa));
   if (a.codes_out)
     DGQ_CUDA_OK(launch_pdl(attn_phase2_kernel<D, NKP, true>, dim3(grid), dim3(AT_THREADS), (size_t)SM2, stream, aa));
@@ -508,12 +876,12 @@ static dgq_status launch_attn(const AttnArgs& a, cudaStream_t stream) {
 }
 
 template <int D>
-static dgq_status launch_attn_d(const AttnArgs& a, cudaStream_t stream) {
-  if (a.nk <= 80) return launch_attn<D, 5>(a, stream);
-  return launch_attn<D, 8>(a, stream);
+static dgq_status launch_attn_d(const AttnArgs& a, bool allow_fused, cudaStream_t stream) {
+  if (a.nk <= 80) return launch_attn<D, 5>(a, allow_fused, stream);
+  return launch_attn<D, 8>(a, allow_fused, stream);
 }
 
-// One partial maximum per phase-1 CTA; the bound holds for every kernel configuration (128 or 256 rows per CTA).
+// One partial maximum per CTA; the bound holds for every kernel configuration (128 or 256 rows per CTA).
 static size_t attn_part_bytes(int B, int H, int nq) {
   return ((size_t)B * H * ((nq + 127) / 128) * sizeof(float) + 255) / 256 * 256;
 }
@@ -543,7 +911,7 @@ static dgq_status attn_check_args(const void* Q, const void* K, const void* V, i
 static dgq_status attn_run(const void* Q, const void* K, const void* V, int B, int H, int nq, int nk, int d,
                            int score_bits, int scale_gran, const float* fixed_scale, int v_bits, void* O,
                            float* scale_out, uint8_t* codes_out, void* workspace, size_t workspace_bytes,
-                           void* stream) {
+                           bool allow_fused, void* stream) {
   dgq_status chk = attn_check_args(Q, K, V, B, H, nq, nk, d, score_bits, scale_gran, v_bits, O);
   if (chk != DGQ_OK) return chk;
   size_t need = 0;
@@ -572,11 +940,11 @@ static dgq_status attn_run(const void* Q, const void* K, const void* V, int B, i
   a.n_row_blocks = 0;  // set per kernel configuration at launch
   cudaStream_t st = (cudaStream_t)stream;
   switch (d) {
-    case 40: return launch_attn_d<40>(a, st);
-    case 64: return launch_attn_d<64>(a, st);
-    case 80: return launch_attn_d<80>(a, st);
-    case 128: return launch_attn_d<128>(a, st);
-    default: return launch_attn_d<160>(a, st);
+    case 40: return launch_attn_d<40>(a, allow_fused, st);
+    case 64: return launch_attn_d<64>(a, allow_fused, st);
+    case 80: return launch_attn_d<80>(a, allow_fused, st);
+    case 128: return launch_attn_d<128>(a, allow_fused, st);
+    default: return launch_attn_d<160>(a, allow_fused, st);
   }
 }
 }  // namespace dgq
@@ -586,7 +954,7 @@ extern "C" dgq_status dgq_cross_attn_logq(const void* Q, const void* K, const vo
                                           float* scale_out, uint8_t* codes_out, void* workspace,
                                           size_t workspace_bytes, void* stream) {
   return dgq::attn_run(Q, K, V, B, H, nq, nk, d, score_bits, scale_gran, fixed_scale, 0, O, scale_out, codes_out,
-                       workspace, workspace_bytes, stream);
+                       workspace, workspace_bytes, true, stream);
 }
 
 extern "C" dgq_status dgq_cross_attn_logq_qv(const void* Q, const void* K, const void* V, int B, int H, int nq,
@@ -595,5 +963,5 @@ extern "C" dgq_status dgq_cross_attn_logq_qv(const void* Q, const void* K, const
                                              void* workspace, size_t workspace_bytes, void* stream) {
   if (v_bits < 2 || v_bits > 8) return DGQ_ERR_INVALID_ARG;
   return dgq::attn_run(Q, K, V, B, H, nq, nk, d, score_bits, scale_gran, fixed_scale, v_bits, O, scale_out,
-                       codes_out, workspace, workspace_bytes, stream);
+                       codes_out, workspace, workspace_bytes, true, stream);
 }

@@ -47,8 +47,9 @@ extern "C" dgq_status dgq_cross_attn_logq_noalloc(const void* Q, const void* K, 
   }
   // The first kernel of the workspace path writes every partial maximum and every row statistic
   // that the second one reads, so stale contents from an earlier call are harmless.
-  return dgq_cross_attn_logq(Q, K, V, B, H, nq, nk, d, score_bits, scale_gran, fixed_scale, O, scale_out,
-                             codes_out, scratch, (size_t)DGQ_NOALLOC_SCRATCH_BYTES, stream);
+  // (always the two-kernel form, which has no launch requirement beyond an ordinary kernel's)
+  return dgq::attn_run(Q, K, V, B, H, nq, nk, d, score_bits, scale_gran, fixed_scale, 0, O, scale_out, codes_out,
+                       scratch, (size_t)DGQ_NOALLOC_SCRATCH_BYTES, false, stream);
 }
 
 namespace dgq {
