@@ -438,8 +438,7 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // The loop is kept lean on purpose: with one convert and half a packed multiply-add per
     // element and group, bookkeeping instructions would otherwise outnumber the arithmetic.
     constexpr int CW = BN / (GEMM_EPI_WARPS / 4);  // columns per thread
-    constexpr int HC = CW / 2;                     // columns per chunk: a group is drained in two
-    static_assert(HC % 8 == 0, "chunk must be whole 8-column loads");
+    static_assert(CW % 8 == 0, "whole 8-column loads and 16-byte output pieces");
     const int q = warp & 3, sl = warp >> 2;
     const int r_tile = q * 32 + lane;  // row inside the tile = TMEM lane
     const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(sl * CW);
@@ -465,21 +464,17 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       pre_s = __ldg(srow);
       pre_z = use_zp ? __ldg(zrow) : 0;
     };
-    // Two register buffers of one chunk each: while the arithmetic runs on one, the tensor-memory
-    // loads of the next chunk (of this group, or of the next group, or of the next tile's first
-    // group) are already in flight into the other.
-    uint32_t rb0[HC], rb1[HC];
-    auto load_chunk = [&](uint32_t taddr, uint32_t(&rb)[HC]) {
+    // One group per round: the warp waits for the group's accumulator, brings its CW columns into registers,
+    // hands the accumulator back to the issuer and then does the arithmetic, while the other epilogue warp of
+    // the scheduler is in another part of its own round.
+    uint32_t rb[CW];
+    auto load_group = [&](uint32_t taddr) {
 #pragma unroll
-      for (int k = 0; k < HC / 16; ++k) tmem_ld16(taddr + k * 16, reinterpret_cast<uint32_t(&)[16]>(rb[k * 16]));
-      if (HC % 16) tmem_ld8(taddr + (HC / 16) * 16, reinterpret_cast<uint32_t(&)[8]>(rb[(HC / 16) * 16]));
+      for (int k = 0; k < CW / 32; ++k) tmem_ld32(taddr + k * 32, reinterpret_cast<uint32_t(&)[32]>(rb[k * 32]));
+      if ((CW % 32) >= 16) tmem_ld16(taddr + (CW / 32) * 32, reinterpret_cast<uint32_t(&)[16]>(rb[(CW / 32) * 32]));
+      if (CW % 16) tmem_ld8(taddr + (CW / 16) * 16, reinterpret_cast<uint32_t(&)[8]>(rb[(CW / 16) * 16]));
     };
-    if ((int)blockIdx.x < n_tiles) {
-      prefetch_tile(blockIdx.x);
-      mbar_wait_lean(full0, 0u, abort_flag);
-      tc_fence_after();
-      load_chunk(t_lane, rb0);
-    }
+    if ((int)blockIdx.x < n_tiles) prefetch_tile(blockIdx.x);
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tile_it) {
       const float* srow_t = srow;
       const int32_t* zrow_t = zrow;
@@ -493,40 +488,28 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int g = 0; g < G; ++g) {
         const float s = s_next;
         const int Z = z_next;
-        const bool more = g + 1 < G || more_tiles;  // another group follows this one
         if (g + 1 < G) {
           s_next = __ldg(srow_t + g + 1);
           if (use_zp) z_next = __ldg(zrow_t + g + 1);
         } else if (more_tiles) {
           prefetch_tile(tile + gridDim.x);
         }
-        const uint32_t taddr = t_lane + ab * (uint32_t)BN;
         uint32_t nab = ab + 1, npar = acc_par;
         if (nab == (uint32_t)NACC) {
           nab = 0;
           npar ^= 1u;
         }
         const unsigned long long s2 = pack_f32x2(s, s);
-        // first chunk: its loads were issued during the previous chunk's arithmetic
+        mbar_wait_lean(full0 + ab * 8u, acc_par, abort_flag);
+        tc_fence_after();
+        load_group(t_lane + ab * (uint32_t)BN);
         tmem_ld_wait();
-        load_chunk(taddr + HC, rb1);
-        // poll the next group's accumulator now, look at the answer after the arithmetic
-        const uint32_t next_ready = more ? mbar_test_addr(full0 + nab * 8u, npar) : 1u;
-#pragma unroll
-        for (int i = 0; i < HC / 2; ++i) cvt_fma_f32x2(y2[i], s2, rb0[2 * i], rb0[2 * i + 1]);
-        if (!next_ready) mbar_wait_lean(full0 + nab * 8u, npar, abort_flag);
-        // second chunk: the accumulator goes back to the issuer as soon as its last columns are in
-        // registers, and the next group's first chunk is requested before the arithmetic
-        tmem_ld_wait();
+        // the accumulator goes back to the issuer as soon as its columns are in registers
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive_addr(empty0 + ab * 8u);
-        if (more) {
-          tc_fence_after();
-          load_chunk(t_lane + nab * (uint32_t)BN, rb0);
-        }
 #pragma unroll
-        for (int i = 0; i < HC / 2; ++i) cvt_fma_f32x2(y2[HC / 2 + i], s2, rb1[2 * i], rb1[2 * i + 1]);
+        for (int i = 0; i < CW / 2; ++i) cvt_fma_f32x2(y2[i], s2, rb[2 * i], rb[2 * i + 1]);
         ab = nab;
         acc_par = npar;
         if (use_zp) {
