@@ -209,10 +209,15 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   reg_dealloc<gemm_regs_other(W4)>();
   if (warp == GEMM_WARP_TMA) {
     // ------------------------------------------------------------ TMA producer
-    // One lane runs the loop; the others go straight to the CTA's final barrier.
-    if (lane == 0) {
-      tma_prefetch_desc(&tmA);
-      if (!W4) tma_prefetch_desc(&tmB);
+    // Five lanes run the loop together and issue their copies with one instruction: lanes 0-3 an A box each
+    // (a conv stage is four boxes, one per atom; a linear stage is one box, lane 0's), lane 4 the B box.
+    // Handing a box to the copy engine costs a thread a few hundred cycles of issue time, which one lane
+    // alone cannot hide when the boxes are as small as a conv atom's.  The other lanes go straight to the
+    // CTA's final barrier.
+    if (lane < 5) {
+      constexpr uint32_t PROD_MASK = 0x1Fu;
+      if (lane == 0) tma_prefetch_desc(&tmA);
+      if (!W4 && lane == 4) tma_prefetch_desc(&tmB);
       const uint32_t empty0 = smem_u32(&sh->empty[0]);
       uint32_t s = 0, empty_par = 1;  // fresh barriers pass a wait for parity 1
       for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
@@ -231,17 +236,18 @@ gq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const int atoms_here = min(4, n_atoms - ks * 4);
           uint32_t bytes = W4 ? 0u : (uint32_t)Cfg::B_STAGE;
           bytes += CONV ? (uint32_t)(atoms_here * 4096) : (uint32_t)GEMM_A_STAGE;
-          mbar_arrive_expect_tx(&sh->full[s], bytes);
+          if (lane == 0) mbar_arrive_expect_tx(&sh->full[s], bytes);  // before any of the copies below
+          __syncwarp(PROD_MASK);
           if (CONV) {
-            for (int j = 0; j < atoms_here; ++j) {
-              const uint32_t e = conv_tab[ks * 4 + j];
-              tma_load_4d(smA + s * GEMM_A_STAGE + j * 4096, &tmA, &sh->full[s], (int)(e & 0xFFFFu),
+            if (lane < atoms_here) {
+              const uint32_t e = conv_tab[ks * 4 + lane];
+              tma_load_4d(smA + s * GEMM_A_STAGE + lane * 4096, &tmA, &sh->full[s], (int)(e & 0xFFFFu),
                           cw + (int)((e >> 16) & 3u) - 1, chh + (int)((e >> 18) & 3u) - 1, cn);
             }
-          } else {
+          } else if (lane == 0) {
             tma_load_2d(smA + s * GEMM_A_STAGE, &tmA, &sh->full[s], ks * 128, m0);
           }
-          if (!W4) tma_load_2d(smB + s * Cfg::B_STAGE, &tmB, &sh->full[s], ks * 128, n0);
+          if (!W4 && lane == 4) tma_load_2d(smB + s * Cfg::B_STAGE, &tmB, &sh->full[s], ks * 128, n0);
           if (++s == (uint32_t)STAGES) {
             s = 0;
             empty_par ^= 1u;
