@@ -64,13 +64,12 @@ __global__ void __launch_bounds__(QA_THREADS, 4) quantize_act_kernel(const Quant
   pdl_launch_dependents();
   for (int i = threadIdx.x; i < head / 16; i += QA_THREADS)
     reinterpret_cast<uint4*>(smem_raw)[i] = __ldg(reinterpret_cast<const uint4*>(a.head) + i);
-  pdl_wait();  // the layout tables above are constants of the grouping; the rows may come from the previous kernel
-  __syncthreads();
   // The row buffers start as NaN everywhere: every row overwrites the positions of its channels, the
   // padding positions are never written again.
   for (int i = lane; i < rpw * a.K_pad / 8; i += 32)
     reinterpret_cast<uint4*>(rows_s)[i] = make_uint4(0x7FFF7FFFu, 0x7FFF7FFFu, 0x7FFF7FFFu, 0x7FFF7FFFu);
-  __syncwarp();
+  __syncthreads();
+  pdl_wait();  // everything above reads only constants of the grouping; the rows may come from the previous kernel
 
   const int vec_per_row = a.C >> 3;
   const float Lf = (float)((1 << a.bits) - 1);
