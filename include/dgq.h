@@ -159,7 +159,9 @@ dgq_status dgq_weight_export(const dgq_weight* w, int8_t* wq, float* sw);
  * there, once per call instead of once per row tile; the bytes stay in L2).
  * Contents undefined on entry and exit; calls that may overlap on the GPU need
  * separate workspaces unless they use the same weight.  NULL / 0 for 8-bit
- * weights.
+ * weights.  NULL with 4-bit weights is allowed: the GEMM then expands the
+ * weights itself, stage by stage and once per row tile (slower); a non-NULL
+ * workspace that is too small is an error.
  * Errors: INVALID_ARG, ALIGNMENT, NOT_CALIBRATED, WORKSPACE, UNSUPPORTED (K_pad *
  * 255 * 127 would overflow int32; more column blocks of 64-128 outputs than the
  * GPU has SMs; conv shape outside the supported tiling), CUDA. */
@@ -180,6 +182,10 @@ dgq_status dgq_linear_workspace_bytes(const dgq_groups* g, const dgq_weight* w, 
  * (dev u8 [B, H, nq, nk-1]) are optional outputs.
  * workspace: dev, at least dgq_cross_attn_workspace_bytes(); contents undefined
  * on entry.  d a multiple of 8, d <= 160, 2 <= nk <= 128.
+ * One kernel: with a dynamic scale its thread blocks exchange their maxima
+ * through the workspace and meet at a grid barrier, so it is launched
+ * cooperatively (and, inside a stream capture, becomes a cooperative kernel
+ * node); grids larger than one resident wave run as two ordinary kernels.
  * Errors: INVALID_ARG (nk < 2), ALIGNMENT, UNSUPPORTED, WORKSPACE, CUDA. */
 dgq_status dgq_cross_attn_logq(const void* Q, const void* K, const void* V, int B, int H, int nq, int nk,
                                int d, int score_bits, int scale_gran, const float* fixed_scale, void* O,

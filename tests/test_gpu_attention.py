@@ -53,6 +53,15 @@ def test_shapes(B, H, nq, nk, d):
     _compare(torch, b, Q, K, V, 8)
 
 
+@pytest.mark.parametrize("gran", [0, 2])
+def test_grid_beyond_one_resident_wave(gran):
+    """8 x 16 heads x 3 row blocks = 384 thread blocks do not fit the device at once (2 per SM), so the call
+    cannot meet at a grid barrier and takes its two-kernel route; same checks as everywhere."""
+    torch, b = gpu()
+    Q, K, V = synth.attention_inputs(12, 8, 16, 768, 77, 40, ctx_dim=64)
+    _compare(torch, b, Q, K, V, 8, gran=gran)
+
+
 @pytest.mark.parametrize("gran", [0, 1, 2])
 def test_scale_granularity(gran):
     torch, b = gpu()
